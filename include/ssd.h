@@ -158,8 +158,9 @@ int ssd_accept_tree(ssd_ctx *ctx, const float *logits, const float *draft_probs,
  * counterpart: this is a deployment variant of ssd_accept_tree.)
  *
  * Who needs it: a serving loop that must never hit the device-wide synchronisation cudaMalloc
- * implies, a thread that is in the middle of a stream capture (where allocation calls are
- * illegal), or a process whose whole memory budget is owned by another allocator.  This entry
+ * implies, or a process whose whole memory budget is owned by another allocator (a framework's
+ * caching pool, a fixed arena handed out at start-up), where a cudaMalloc from a library would
+ * either fail or take memory that allocator counts on.  This entry
  * point needs no ssd_ctx and calls no allocation routine, on the device or on the host: its
  * scratch (the fp64 residual distribution of the sampling rule, and a few small arrays) lives in
  * fixed device arrays that every GPU loading the library holds until the process exits
@@ -172,7 +173,8 @@ int ssd_accept_tree(ssd_ctx *ctx, const float *logits, const float *draft_probs,
  * context would otherwise supply.  logits / draft_probs are DEVICE pointers, everything else host.
  *
  * The first call on a device looks up the arrays' device addresses (cudaGetSymbolAddress); make
- * that first call outside any stream capture.  All calls share the same arrays: they keep the
+ * that first call before any stream capture begins.  `cuda_stream` itself must not be capturing: the
+ * call copies its few result words back and waits for the stream.  All calls share the same arrays: they keep the
  * previous call's contents (nothing in them has to start at zero - every word a call reads it has
  * written first), and two calls whose kernels overlap on the GPU (different streams or threads)
  * race on them, so serialise such calls.  Waits for the stream before returning.

@@ -20,6 +20,7 @@ def _run(name, P, trees, seed=0, chunk=256, persistent=False):
     import paper_2308_04623_b200 as ssd
     p = gpu_util.Pair(name, seed=seed)
     worst = {}
+    fragile = 0
     try:
         if persistent:
             p.ctx.set_tuning(ssd.SSD_TUNE_PERSISTENT, 1)
@@ -44,7 +45,11 @@ def _run(name, P, trees, seed=0, chunk=256, persistent=False):
                                               top_k=top_k, rng=srng)
                 opath, onxt, margin = ssd_oracle.accept_tree(got.astype(np.float32), draft, tokens, parent, mode=1, temperature=1.0,
                                                              top_k=top_k, seed=11, step=5)
-                assert (path, nxt) == (opath, onxt) or margin < 1e-9, (label, top_k, margin)
+                if (path, nxt) != (opath, onxt):
+                    assert margin < 1e-9, (label, top_k, margin)
+                    fragile += 1
+        print("draws forgiven for a margin below 1e-9:", fragile)
+        assert fragile == 0
         assert p.ctx.device_status() == 0
     finally:
         p.close()

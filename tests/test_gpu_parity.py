@@ -172,15 +172,21 @@ def test_sampling_walk_goes_deep_and_matches(tiny):
         mix = 0.7 * probs[parent[c]] + 0.3 * rng.dirichlet(np.full(V, 0.5))
         draft[c] = mix.astype(np.float32)
         tokens[c] = rng.choice(V, p=mix / mix.sum())
-    deep = 0
+    deep = fragile = 0
     for step in range(300):
         got, want, margin = _accept_both(p, logits, draft, tokens, parent, 1, 7, step)
-        assert got == want or margin < 1e-9, (step, got, want, margin)
+        if got != want:
+            assert margin < 1e-9, (step, got, want, margin)
+            fragile += 1
         deep += len(want[0]) > 2
     assert deep > 20
     for step in range(100):  # top-k and temperature warp
         got, want, margin = _accept_both(p, logits, draft, tokens, parent, 1, 9, step, temperature=0.7, top_k=50)
-        assert got == want or margin < 1e-9, (step, got, want, margin)
+        if got != want:
+            assert margin < 1e-9, (step, got, want, margin)
+            fragile += 1
+    print("draws forgiven for a margin below 1e-9:", fragile)
+    assert fragile == 0
 
 
 def test_accept_special_rows(tiny):
@@ -221,6 +227,7 @@ def test_sampling_at_a_large_vocabulary_star_tree_ties_and_long_support(ssd):
         tied[:, rng.choice(V, size=3000, replace=False)] = 9.0   # 3000 ties at the top: any k <= 3000 keeps them all
         draft = ssd_synth.draft_rows_gamma(n, V, rng)
         lg_dev, tied_dev, dp_dev = (torch.from_numpy(a).cuda() for a in (logits, tied, draft))
+        fragile = 0
         for lg_np, lg_d, top_k in ((logits, lg_dev, 0), (logits, lg_dev, 50), (logits, lg_dev, 1000), (tied, tied_dev, 50), (tied, tied_dev, 0)):
             for step in range(3):
                 srng = ssd.binding.ssd_rng(5, step)
@@ -228,7 +235,11 @@ def test_sampling_at_a_large_vocabulary_star_tree_ties_and_long_support(ssd):
                                       top_k=top_k, rng=srng)
                 opath, onxt, margin = ssd_oracle.accept_tree(lg_np, draft, tokens, parent, mode=1, temperature=1.0, top_k=top_k,
                                                              seed=5, step=step, max_nodes=cfg["max_nodes"])
-                assert got == (opath, onxt) or margin < 1e-9, (top_k, step, margin)
+                if got != (opath, onxt):
+                    assert margin < 1e-9, (top_k, step, margin)
+                    fragile += 1
+        print("draws forgiven for a margin below 1e-9:", fragile)
+        assert fragile == 0
     finally:
         ctx.close()
 
@@ -295,6 +306,34 @@ def test_commit_moves_exactly_the_path_rows(tiny):
             assert np.array_equal(after[:5], before[l][w][:5])
             for j, c in enumerate(path):
                 assert np.array_equal(after[5 + j], before[l][w][5 + c])
+
+
+@pytest.mark.parametrize("path", [[0, 2, 5, 12], [0], [0, 1, 3, 7, 15, 31]])
+def test_bf16_commit_moves_exactly_the_path_rows(path, util):
+    """The same bit-exact gather on the bf16 cache, whose V is stored transposed and moved by a kernel of its own:
+    K and V scratch rows are read before the commit and must sit, bit for bit, at their committed slots after it; the
+    prefix rows stay as they were.  (An odd prefix length, so that pairs of transposed-V keys straddle slots.)"""
+    p = util.Pair("ragged_bf16", seed=4)
+    try:
+        rng = np.random.default_rng(12)
+        P = 37
+        p.prefill(ssd_synth.uniform_tokens(P, p.V, rng), chunk=32)
+        parent = ssd_synth.tree_complete_binary(5)  # 63 nodes; [0, 1, 3, 7, 15, 31] is its leftmost path
+        n = len(parent)
+        p.verify(ssd_synth.uniform_tokens(n, p.V, rng), parent)
+        L = p.cfg["n_layer"]
+        before = [[p.ctx.kv_read(p.kv, l, w, 0, P + n) for w in (0, 1)] for l in range(L)]
+        p.commit(path)
+        assert len(p.kv) == P + len(path)
+        for l in range(L):
+            for w in (0, 1):
+                after = p.ctx.kv_read(p.kv, l, w, 0, P + len(path))
+                assert np.array_equal(after[:P], before[l][w][:P])
+                for j, c in enumerate(path):
+                    assert np.array_equal(after[P + j], before[l][w][P + c]), (l, w, j, c)
+                assert np.abs(after).max() > 0
+    finally:
+        p.close()
 
 
 # --------------------------------------------------------------------------- errors
@@ -435,9 +474,10 @@ def test_bf16_steps_with_commit(util):
             root = nxt
             # committed rows: bf16 storage of the fp32 projections, compared with the oracle's exact rows
             for l in range(p.cfg["n_layer"]):
-                a = p.ctx.kv_read(p.kv, l, 0, 0, len(p.kv))
-                b = p.okv.read(l, 0, 0, len(p.kv))
-                assert np.abs(a - b).max() <= 3e-2
+                for which_kv in (0, 1):
+                    a = p.ctx.kv_read(p.kv, l, which_kv, 0, len(p.kv))
+                    b = p.okv.read(l, which_kv, 0, len(p.kv))
+                    assert np.abs(a - b).max() <= 3e-2
     finally:
         p.close()
 

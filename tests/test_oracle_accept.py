@@ -368,3 +368,68 @@ def test_non_finite_logits_are_reported():
     with pytest.raises(ssd_oracle.OracleError) as e:
         ssd_oracle.accept_tree(lg, None, [0, 1], [-1, 0], mode=0)
     assert e.value.code == ssd_oracle.ORC_BAD_ARG
+
+
+def test_min_margin_closed_form_on_four_word_vocabulary():
+    """The margin the oracle reports (how close the nearest decision came to flipping) on a hand-made case
+    where every quantity is a dyadic rational, so the expected value is exact in fp64.
+
+    Vocabulary of 4, all logits zero: every node's target law is (1/4, 1/4, 1/4, 1/4).  One child c = 1 of
+    the root with token 0, proposed from q = (1/2, 1/2, 0, 0).  With u = u(seed, step, 2c):
+      accept test   u / 2 < 1 / 4, relative distance |u / 2 - 1 / 4| / (1 / 4) = |2 u - 1|;
+      accepted      the extra token is drawn at the leaf from the uniform law with u' = u(seed, step, 2 c + 1):
+                    cell v = floor(4 u'), distance to the nearer cell edge over the cell's mass
+                    = min(4 u' - v, v + 1 - 4 u');
+      refused       residual = positive part of p - q = (0, 0, 1/4, 1/4), renormalised (0, 0, 1/2, 1/2); the
+                    extra token is drawn at the root with u' = u(seed, step, 1): token 2 if u' < 1 / 2 else 3,
+                    distance min(2 u' - (v - 2), (v - 1) - 2 u').
+    The reported margin is the smaller of the two distances."""
+    V = 4
+    logits = np.zeros((2, V), dtype=np.float32)
+    draft = np.zeros((2, V), dtype=np.float32)
+    draft[1] = [0.5, 0.5, 0.0, 0.0]
+    tokens, parent = [3, 0], [-1, 0]
+    seen = {"accepted": 0, "refused": 0}
+    for step in range(64):
+        u = ssd_oracle.uniform(123, step, 2)
+        path, nxt, margin = ssd_oracle.accept_tree(logits, draft, tokens, parent, mode=1, seed=123, step=step)
+        m1 = abs(2.0 * u - 1.0)
+        if u < 0.5:
+            u2 = ssd_oracle.uniform(123, step, 3)
+            v = int(np.floor(4.0 * u2))
+            m2 = min(4.0 * u2 - v, v + 1 - 4.0 * u2)
+            assert (path, nxt) == ([0, 1], v)
+            seen["accepted"] += 1
+        else:
+            u2 = ssd_oracle.uniform(123, step, 1)
+            v = 2 if u2 < 0.5 else 3
+            m2 = min(2.0 * u2 - (v - 2), (v - 1) - 2.0 * u2)
+            assert (path, nxt) == ([0], v)
+            seen["refused"] += 1
+        assert abs(margin - min(m1, m2)) <= 1e-12, (step, margin, m1, m2)
+        assert margin > 1e-6  # none of these 24-bit draws sits on a threshold
+    assert seen["accepted"] >= 10 and seen["refused"] >= 10
+
+
+def test_min_margin_shrinks_to_the_distance_of_a_near_threshold_draw():
+    """A proposal probability chosen so that u * q[x] misses r[x] by a known relative amount: the oracle must
+    report exactly that amount (a margin that came out too small would make the parity tests forgive real
+    mismatches, one that came out too large would hide fragile draws)."""
+    V = 4
+    logits = np.zeros((2, V), dtype=np.float32)
+    tokens, parent = [3, 0], [-1, 0]
+    for step, eps in ((0, 2.0 ** -20), (1, -2.0 ** -20), (2, 2.0 ** -12)):
+        u = ssd_oracle.uniform(9, step, 2)
+        q0 = np.float32(0.25 * (1.0 + eps) / u)          # u * q0 = (1 + eps) / 4 up to the rounding of q0 to fp32
+        if not (0.0 < q0 <= 1.0):
+            continue
+        draft = np.zeros((2, V), dtype=np.float32)
+        draft[1] = [q0, 1.0 - q0, 0.0, 0.0]
+        path, nxt, margin = ssd_oracle.accept_tree(logits, draft, tokens, parent, mode=1, seed=9, step=step)
+        rel = abs(u * float(q0) - 0.25) / 0.25           # with the fp32 value of q0 the oracle was given
+        assert len(path) == (2 if u * float(q0) < 0.25 else 1)
+        assert margin <= rel + 1e-15
+        if margin < rel - 1e-15:                          # then the extra draw was the closer call
+            assert margin >= 0.0
+        else:
+            assert abs(margin - rel) <= 1e-15

@@ -1,11 +1,14 @@
 """The allocation-free acceptance entry point against the regular one (GPU, through the C ABI).
 
-Some callers cannot allocate device memory at the moment they need an acceptance walk - a thread
-inside a stream capture, a latency-critical serving loop that must not trigger the implicit
-synchronisation of an allocation, a process whose memory is owned by another allocator.  For them
-``ssd_accept_tree_noalloc`` keeps its scratch in fixed device arrays of the library.  This file is
-named so that pytest collects it last: if it fails, every other test has already run.  It passes both
-alone in a fresh process and after the rest of the suite.
+Some callers cannot allocate device memory at the moment they need an acceptance walk - a
+latency-critical serving loop that must not trigger the implicit synchronisation of an allocation, a
+process whose memory is owned by another allocator (a caching pool, a fixed arena), where a library's
+own cudaMalloc would fail or take memory that allocator counts on.  For them
+``ssd_accept_tree_noalloc`` keeps its scratch in fixed device arrays of the library.  The results are
+compared with the regular entry point AND with the CPU oracle (the single-CTA walk kernel behind this
+entry point is not reached by any other test), and the free device memory is checked not to move across
+the calls.  This file is named so that pytest collects it last: if it fails, every other test has
+already run.  It passes both alone in a fresh process and after the rest of the suite.
 """
 import ctypes as C
 
@@ -14,6 +17,7 @@ import pytest
 import torch
 
 import ssd_synth
+from oracle import ssd_oracle
 
 pytestmark = pytest.mark.gpu
 
@@ -49,7 +53,7 @@ def test_noalloc_entry_point_matches_regular_entry_point_twice_in_a_row(V):
         rng = np.random.default_rng(V)
         parent = ssd_synth.tree_branching(24, (3, 2, 2, 1, 1))
         n = len(parent)
-        calls = 0
+        calls = fragile = 0
         for rep in range(2):  # two calls in a row per setting: the shared scratch keeps the previous call's contents
             logits = (rng.normal(size=(n, V)) * 2.5).astype(np.float32)
             probs = np.exp(logits.astype(np.float64))
@@ -62,14 +66,26 @@ def test_noalloc_entry_point_matches_regular_entry_point_twice_in_a_row(V):
                 tokens[c] = rng.choice(V, p=mix / mix.sum())
             lg = torch.from_numpy(logits).cuda()
             dp = torch.from_numpy(draft).cuda()
+            # one warm call (symbol look-up, lazy module load), then the free device memory must not move
+            _call_noalloc(ssd, lg, dp, tokens, parent, V, ssd.SSD_SAMPLING, 1, 0, 1.0, 0)
+            torch.cuda.synchronize()
+            free_before = torch.cuda.mem_get_info()[0]
             for mode, T, k in ((ssd.SSD_GREEDY, 1.0, 0), (ssd.SSD_SAMPLING, 1.0, 0), (ssd.SSD_SAMPLING, 0.75, 50)):
                 for step in range(6):
                     want = _call_regular(ssd, ctx, lg, dp, tokens, parent, mode, 11, step, T, k)
                     rc, path, nxt, new_step = _call_noalloc(ssd, lg, dp, tokens, parent, V, mode, 11, step, T, k)
                     assert rc == ssd.SSD_OK
                     assert (path, nxt, new_step) == want  # integer results: exact
+                    opath, onxt, margin = ssd_oracle.accept_tree(logits, draft if mode else None, tokens, parent, mode=mode,
+                                                                 temperature=float(np.float32(T)), top_k=k, seed=11, step=step)
+                    if (path, nxt) != (opath, onxt):
+                        assert margin < 1e-9, (mode, T, k, step, margin)
+                        fragile += 1
                     calls += 1
+            torch.cuda.synchronize()
+            assert torch.cuda.mem_get_info()[0] == free_before  # nothing was allocated on the device
         assert calls == 36
+        assert fragile == 0
     finally:
         ctx.close()
 
