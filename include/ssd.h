@@ -201,31 +201,31 @@ int ssd_kv_read(ssd_ctx *ctx, const ssd_kv *kv, int32_t layer, int32_t which, in
  * Performance knobs of the bf16 path (defaults in brackets); results stay within the stated
  * tolerances for every setting.  Waits for the stream and drops the captured graphs.
  *   SSD_TUNE_LOW_PLANE [1]        feed activations to the tensor cores as bf16 hi + lo pairs
+ *   SSD_TUNE_ATTN_LOW_PLANE [0]   the same for the queries and softmax weights inside the attention kernel (off: one bf16 value each,
+ *                                 which rounds them as coarsely as the bf16 cache already rounds K and V; 6.5e-3 -> 7.4e-3 maximum logit
+ *                                 error at the GPT-2-large shape, 30 us per step faster)
  *   SSD_TUNE_DEPENDENT_LAUNCH [1] programmatic dependent launch between the forward's kernels
  *   SSD_TUNE_GRAPH [1]            replay one captured CUDA graph per tree size
- *   SSD_TUNE_GEMM_CTAS [0]        CTAs per projection kernel of the layers; 0 = choose (two per SM for trees of <= 64 nodes, else one)
+ *   SSD_TUNE_GEMM_CTAS [0]        CTAs per projection kernel of the layers; 0 = choose (two per SM for small trees, else one)
+ *   SSD_TUNE_CLUSTER_REDUCE [0]   trees of up to 64 nodes: reduce every projection's split-K partial sums inside a thread-block
+ *                                 cluster and fuse LayerNorm / GELU / residual into its epilogue (5 launches per layer instead
+ *                                 of 8, layers reproducible bit for bit; measured slower than the default so far)
+ *   SSD_TUNE_CLUSTER_MAX [8]      largest cluster (CTAs per output tile) of that path, 1..16
+ *   SSD_TUNE_CLUSTER_QKV / _O / _FC / _PROJ [0]  cluster size of one of the four projections of a layer; 0 = choose
  *   SSD_TUNE_HEAD_CTAS [0]        CTAs of the LM-head projection; 0 = as the layers'
- *   SSD_TUNE_FUSED_TAILS [0]      fold the LayerNorms into the projections and let the CTA that completes an
- *                                 output tile prepare the next operand (5 launches per layer instead of 8; measured slower so far)
  *   SSD_TUNE_KERNEL_TRACE [0]     record a timeline of every kernel of a bf16 forward (see ssd_get_phase_trace)
- *   SSD_TUNE_PERSISTENT [0]       run all layers in one persistent kernel (trees of <= 64 nodes)
- *   SSD_TUNE_SELF_STAGED [0]      the projections behind a LayerNorm or the GELU convert their activations themselves
- *                                 (LayerNorm folded into the consumer; 5 launches per layer instead of 8; measured slower so far);
- *                                 applies when every CTA's share of a projection fits the shared-memory pipeline, else the 8-launch path runs
  */
-enum { SSD_TUNE_LOW_PLANE = 0, SSD_TUNE_DEPENDENT_LAUNCH = 1, SSD_TUNE_GRAPH = 2, SSD_TUNE_GEMM_CTAS = 3, SSD_TUNE_PERSISTENT = 4, SSD_TUNE_FUSED_TAILS = 5,
-       SSD_TUNE_SELF_STAGED = 6, SSD_TUNE_HEAD_CTAS = 7, SSD_TUNE_KERNEL_TRACE = 8 };
+enum { SSD_TUNE_LOW_PLANE = 0, SSD_TUNE_DEPENDENT_LAUNCH = 1, SSD_TUNE_GRAPH = 2, SSD_TUNE_GEMM_CTAS = 3, SSD_TUNE_CLUSTER_REDUCE = 4,
+       SSD_TUNE_CLUSTER_MAX = 5, SSD_TUNE_ATTN_LOW_PLANE = 6, SSD_TUNE_HEAD_CTAS = 7, SSD_TUNE_KERNEL_TRACE = 8, SSD_TUNE_CLUSTER_QKV = 9, SSD_TUNE_CLUSTER_O = 10,
+       SSD_TUNE_CLUSTER_FC = 11, SSD_TUNE_CLUSTER_PROJ = 12 };
 int ssd_set_tuning(ssd_ctx *ctx, int32_t knob, int32_t value);
 
 /*
- * Phase trace of the last forward that ran as the persistent kernel: nanosecond device
- * timestamps taken by one CTA when it finishes the work of a phase and when it leaves the grid
- * barrier that follows (plus one when the row statistics of a LayerNorm arrive).  `out_ns` (host)
- * receives up to `capacity` values, `count` how many.  Waits for the stream.  A profiling aid.
- * With SSD_TUNE_KERNEL_TRACE set (eight-launch bf16 path) the values are instead eight per kernel of the last
- * forward, in launch order after the two set-up kernels' slots: the first CTA's time of entry, of its dependencies
- * being met, of its end and (projections) of its first complete accumulator, then the same four of the last CTA,
- * except that the seventh value is the latest end over all CTAs; unused slots are zero.
+ * Per-kernel timeline of the last bf16 forward run with SSD_TUNE_KERNEL_TRACE set: eight nanosecond device
+ * timestamps per kernel, in launch order: the first CTA's time of entry, of its dependencies being met, of
+ * its end and (projections) of its first complete accumulator, then the same four of the last CTA, except that
+ * the seventh value is the latest end over all CTAs; unused slots are zero.  `out_ns` (host) receives up to
+ * `capacity` values, `count` how many.  Waits for the stream.  A profiling aid.
  */
 int ssd_get_phase_trace(ssd_ctx *ctx, uint64_t *out_ns, int32_t capacity, int32_t *count);
 

@@ -44,7 +44,7 @@ def build(force: bool = False, verbose: bool = False) -> str:
     for src in sources():
         obj = os.path.join(HERE, "build", os.path.basename(src)[:-3] + ".o")
         cmd = [_nvcc()] + NVCC_FLAGS + \
-            (["-Xptxas", "-v"] if verbose else []) + ["-I", INCLUDE, "-I", CSRC, "-c", src, "-o", obj]
+            (["-Xptxas", "-v"] if verbose else []) + os.environ.get("SSD_NVCC_EXTRA", "").split() + ["-I", INCLUDE, "-I", CSRC, "-c", src, "-o", obj]
         procs.append((src, subprocess.Popen(cmd, stdout=subprocess.PIPE, stderr=subprocess.STDOUT, text=True)))
         objs.append(obj)
     failed = False

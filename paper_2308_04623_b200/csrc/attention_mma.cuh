@@ -44,19 +44,6 @@ struct Output {
     int max_nodes, n_head;
 };
 
-// When the QKV projection was computed on x * gain without the LayerNorm's normalisation
-// (persistent kernel), q/k/v = rstd * (acc - mean * c1) + c2 is applied on load: `stats` holds
-// each row's sum and sum of squares of x, c1 = W g and c2 = W beta + b per output feature.
-struct LnFold {
-    const float *stats, *c1, *c2; // null stats = the projections are already final
-    float inv_d, eps;
-};
-__device__ __forceinline__ void row_stats(const LnFold &f, int row, float &mean, float &rstd) {
-    const float2 s = __ldcg(reinterpret_cast<const float2 *>(f.stats + 2 * row));
-    mean = s.x * f.inv_d;
-    rstd = rsqrtf(fmaxf(s.y * f.inv_d - mean * mean, 0.f) + f.eps);
-}
-
 __device__ __forceinline__ void mma_bf16(float (&c)[4], const uint32_t (&a)[4], uint32_t b0, uint32_t b1) {
     asm volatile("mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
                  : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
@@ -86,11 +73,13 @@ struct BlockFrags {
 // registers only when a warp handles several blocks).
 // PDL_WAIT: the item runs in a kernel launched as a programmatic dependent: the committed cache rows of its
 // first blocks (written by earlier steps) are requested first, then it waits for the kernel that produced `qkv`.
-template <int NW, bool PREFETCH, bool PDL_WAIT = false>
+// LO: q and the softmax weights enter the tensor cores as hi + lo pairs (two MMAs each); without it as one bf16 value, which
+// rounds them as coarsely as the cache already rounds K and V.
+template <int NW, bool PREFETCH, bool PDL_WAIT = false, bool LO = true>
 __device__ __forceinline__ void work_item(int tid, int bar_id, unsigned char *smem_raw, int h, int tile0, int split, int n_splits,
                                           bool store_scratch, const float *__restrict__ qkv, const StepInfo *__restrict__ info,
                                           size_t layer_offset, const TreeMeta &meta, int n, int d, int cap, const Output &out,
-                                          const LnFold &fold, unsigned long long *trace = nullptr) {
+                                          unsigned long long *trace = nullptr) {
     const int warp = tid >> 5, lane = tid & 31, g = lane >> 2, t = lane & 3;
     const int P = info->kv_len, Pf = P & ~15, n_keys = P + n;
     const int local_keys = n_keys - Pf;             // keys held in shared memory: prefix tail + tree
@@ -152,13 +141,6 @@ __device__ __forceinline__ void work_item(int tid, int bar_id, unsigned char *sm
         float4 v = make_float4(0.f, 0.f, 0.f, 0.f);
         if (row < n) { // (L2 loads: inside the persistent kernel these values come from other SMs)
             v = __ldcg(reinterpret_cast<const float4 *>(qkv + (size_t)row * 3 * d + h * DH + c));
-            if (fold.stats) {
-                float mean, rstd;
-                row_stats(fold, row, mean, rstd);
-                const float4 c1 = __ldg(reinterpret_cast<const float4 *>(fold.c1 + h * DH + c)), c2 = __ldg(reinterpret_cast<const float4 *>(fold.c2 + h * DH + c));
-                v.x = rstd * (v.x - mean * c1.x) + c2.x; v.y = rstd * (v.y - mean * c1.y) + c2.y;
-                v.z = rstd * (v.z - mean * c1.z) + c2.z; v.w = rstd * (v.w - mean * c1.w) + c2.w;
-            }
         }
         *reinterpret_cast<float4 *>(s_q + r * QROW + c) = v;
     }
@@ -184,21 +166,6 @@ __device__ __forceinline__ void work_item(int tid, int bar_id, unsigned char *sm
                 float4 k0 = __ldcg(reinterpret_cast<const float4 *>(kf)), k1 = __ldcg(reinterpret_cast<const float4 *>(kf + 4));
                 float4 v0 = __ldcg(reinterpret_cast<const float4 *>(vf)), v1 = __ldcg(reinterpret_cast<const float4 *>(vf + 4));
                 float kk[8] = {k0.x, k0.y, k0.z, k0.w, k1.x, k1.y, k1.z, k1.w}, vf8[8] = {v0.x, v0.y, v0.z, v0.w, v1.x, v1.y, v1.z, v1.w};
-                if (fold.stats) {
-                    float mean, rstd;
-                    row_stats(fold, j, mean, rstd);
-                    const float4 a0 = __ldg(reinterpret_cast<const float4 *>(fold.c1 + d + h * DH + c)), a1 = __ldg(reinterpret_cast<const float4 *>(fold.c1 + d + h * DH + c + 4));
-                    const float4 b0 = __ldg(reinterpret_cast<const float4 *>(fold.c2 + d + h * DH + c)), b1 = __ldg(reinterpret_cast<const float4 *>(fold.c2 + d + h * DH + c + 4));
-                    const float4 e0 = __ldg(reinterpret_cast<const float4 *>(fold.c1 + 2 * d + h * DH + c)), e1 = __ldg(reinterpret_cast<const float4 *>(fold.c1 + 2 * d + h * DH + c + 4));
-                    const float4 f0 = __ldg(reinterpret_cast<const float4 *>(fold.c2 + 2 * d + h * DH + c)), f1 = __ldg(reinterpret_cast<const float4 *>(fold.c2 + 2 * d + h * DH + c + 4));
-                    const float kc1[8] = {a0.x, a0.y, a0.z, a0.w, a1.x, a1.y, a1.z, a1.w}, kc2[8] = {b0.x, b0.y, b0.z, b0.w, b1.x, b1.y, b1.z, b1.w};
-                    const float vc1[8] = {e0.x, e0.y, e0.z, e0.w, e1.x, e1.y, e1.z, e1.w}, vc2[8] = {f0.x, f0.y, f0.z, f0.w, f1.x, f1.y, f1.z, f1.w};
-#pragma unroll
-                    for (int q = 0; q < 8; ++q) {
-                        kk[q] = rstd * (kk[q] - mean * kc1[q]) + kc2[q];
-                        vf8[q] = rstd * (vf8[q] - mean * vc1[q]) + vc2[q];
-                    }
-                }
                 kq.x = pack_bf16(kk[0], kk[1]); kq.y = pack_bf16(kk[2], kk[3]); kq.z = pack_bf16(kk[4], kk[5]); kq.w = pack_bf16(kk[6], kk[7]);
 #pragma unroll
                 for (int i = 0; i < 4; ++i) vw[i] = pack_bf16(vf8[2 * i], vf8[2 * i + 1]);
@@ -268,10 +235,10 @@ __device__ __forceinline__ void work_item(int tid, int bar_id, unsigned char *sm
         for (int m = 0; m < 2; ++m) {
             float c[4] = {0.f, 0.f, 0.f, 0.f}, cl[4] = {0.f, 0.f, 0.f, 0.f}; // q's high and low parts: two chains of four, not one of eight
             const uint4 k0 = cur.k[m][0], k1 = cur.k[m][1];
-            mma_bf16(c, qh[0], k0.x, k0.y); mma_bf16(cl, ql[0], k0.x, k0.y);
-            mma_bf16(c, qh[1], k0.z, k0.w); mma_bf16(cl, ql[1], k0.z, k0.w);
-            mma_bf16(c, qh[2], k1.x, k1.y); mma_bf16(cl, ql[2], k1.x, k1.y);
-            mma_bf16(c, qh[3], k1.z, k1.w); mma_bf16(cl, ql[3], k1.z, k1.w);
+            mma_bf16(c, qh[0], k0.x, k0.y); if (LO) mma_bf16(cl, ql[0], k0.x, k0.y);
+            mma_bf16(c, qh[1], k0.z, k0.w); if (LO) mma_bf16(cl, ql[1], k0.z, k0.w);
+            mma_bf16(c, qh[2], k1.x, k1.y); if (LO) mma_bf16(cl, ql[2], k1.x, k1.y);
+            mma_bf16(c, qh[3], k1.z, k1.w); if (LO) mma_bf16(cl, ql[3], k1.z, k1.w);
 #pragma unroll
             for (int q = 0; q < 4; ++q) c[q] += cl[q];
 #pragma unroll
@@ -313,7 +280,7 @@ __device__ __forceinline__ void work_item(int tid, int bar_id, unsigned char *sm
 #pragma unroll
         for (int dt = 0; dt < 8; ++dt) {
             mma_bf16(oacc[dt], ph, cur.v[dt].x, cur.v[dt].y);
-            mma_bf16(oacc[dt], pl, cur.v[dt].x, cur.v[dt].y);
+            if (LO) mma_bf16(oacc[dt], pl, cur.v[dt].x, cur.v[dt].y);
         }
         b = nb;
         if (PREFETCH) {

@@ -44,7 +44,6 @@ constexpr int SMEM_BUDGET_SHARED = 106 * 1024;
 #ifndef EPI_POLL_NS
 #define EPI_POLL_NS 32
 #endif
-constexpr int STAGE_BATCH = 8;              // 16-byte operand chunks a thread converts per round when it stages operand B itself
 
 struct GemmParams {
     float *y;          // [n, ldy] fp32, accumulated into; null = take info->logits
@@ -58,7 +57,6 @@ struct GemmParams {
     int split;         // > 0: every output tile's k tiles are shared by `split` CTAs of its own (grid = split * n_tiles); 0: stream-K ranges
     int use_lo;
     int32_t *status;   // device error word
-    GemmFusion f;      // fused LayerNorm fold / tails (all zero = none)
     unsigned long long *trace; // timeline slots of this launch or null
 };
 
@@ -69,17 +67,9 @@ struct __align__(8) Barriers {
     uint64_t acc_empty[2];
     uint32_t tmem_base;
     uint32_t abort;
-    int tail_last;                // broadcast: this CTA added the last partial sum of the tile
-    float mean[SSD_MAX_NODES], rstd[SSD_MAX_NODES]; // row statistics (fold / GELU tail)
-    float sum1[SSD_MAX_NODES], sum2[SSD_MAX_NODES]; // this CTA's share of the rows' sum / sum of squares (self-staged LayerNorm operand)
 };
 
 __device__ __forceinline__ void epi_sync() { asm volatile("bar.sync 2, 128;" ::: "memory"); } // the four epilogue warps
-
-__device__ __forceinline__ float gelu_tanh_fast(float z) { // 0.5 z (1 + tanh u) = z / (1 + exp(-2u))
-    const float u2 = 1.5957691216057308f * (z + 0.044715f * z * z * z);
-    return __fdividef(z, 1.0f + __expf(-u2));
-}
 
 __device__ __forceinline__ void fail(const GemmParams &p, Barriers *b, int code) {
     atomicExch(p.status, code);
@@ -87,103 +77,8 @@ __device__ __forceinline__ void fail(const GemmParams &p, Barriers *b, int code)
 }
 
 
-// Operand B built by the CTA itself from an fp32 source, so that no separate preparation kernel sits
-// between two projections.  The four epilogue warps convert this CTA's k tiles (one stage per unit, no
-// ring reuse) into the 128-byte-swizzled bf16 hi / lo layout the activation boxes would have had:
-//   SRC_LN_GAIN  B = src * gain.  The LayerNorm in front of the projection is applied by the consumer of
-//                the accumulators as rstd * (acc - mean * c1) + c2; the rows' sum and sum of squares are
-//                contributed by the CTAs holding units of output tile 0 (they cover every k tile once),
-//                which then count themselves on `stats_counter`.
-//   SRC_GELU     B = gelu(src).
-__device__ __forceinline__ void stage_operand(const GemmParams &p, Barriers *bars, uint8_t *smem, int stage_bytes, int b_bytes, int u0, int u1,
-                                              int et, int lane) {
-    const int nu = u1 - u0, cpu = p.n_pad * 8 /* 16-byte chunks per unit */, total = nu * cpu;
-    const bool ln = p.f.src_mode == SRC_LN_GAIN;
-    const bool stats = ln && p.f.stats_out && u0 < p.k_tiles;
-    if (stats) {
-        for (int i = et; i < p.n; i += 128) { bars->sum1[i] = 0.f; bars->sum2[i] = 0.f; }
-        epi_sync();
-    }
-    int signalled = 0;
-    for (int base = 0; base < total; base += 128 * STAGE_BATCH) {
-        float4 v[STAGE_BATCH][2];
-        // (n_pad is a multiple of 16, so a block of 128 chunks lies inside one unit and inside `total`, or outside it)
-#pragma unroll
-        for (int b = 0; b < STAGE_BATCH; ++b) {
-            const int q = base + b * 128 + et;
-            v[b][0] = v[b][1] = make_float4(0.f, 0.f, 0.f, 0.f);
-            if (q < total) {
-                const int j = q / cpu, r = q - j * cpu, i = r >> 3, c = r & 7, kt = (u0 + j) % p.k_tiles;
-                if (i < p.n) {
-                    const float4 *s4 = reinterpret_cast<const float4 *>(p.f.src + (size_t)i * p.f.src_ld + kt * TILE_K + c * 8);
-                    v[b][0] = __ldcg(s4);
-                    v[b][1] = __ldcg(s4 + 1);
-                }
-            }
-        }
-#pragma unroll
-        for (int b = 0; b < STAGE_BATCH; ++b) {
-            const int q = base + b * 128 + et;
-            if (q < total) {
-                const int j = q / cpu, r = q - j * cpu, i = r >> 3, c = r & 7, u = u0 + j, kt = u % p.k_tiles;
-                float a[8] = {v[b][0].x, v[b][0].y, v[b][0].z, v[b][0].w, v[b][1].x, v[b][1].y, v[b][1].z, v[b][1].w};
-                if (ln) {
-                    if (stats && u < p.k_tiles) { // the same for all 128 threads
-                        float s1 = 0.f, s2 = 0.f;
-#pragma unroll
-                        for (int t = 0; t < 8; ++t) { s1 += a[t]; s2 += a[t] * a[t]; }
-#pragma unroll
-                        for (int off = 1; off < 8; off <<= 1) { // the eight lanes that share a row
-                            s1 += __shfl_xor_sync(0xffffffffu, s1, off);
-                            s2 += __shfl_xor_sync(0xffffffffu, s2, off);
-                        }
-                        if ((lane & 7) == 0 && i < p.n) { atomicAdd(&bars->sum1[i], s1); atomicAdd(&bars->sum2[i], s2); }
-                    }
-                    const float4 *g4 = reinterpret_cast<const float4 *>(p.f.gain + kt * TILE_K + c * 8);
-                    const float4 g0 = __ldg(g4), g1 = __ldg(g4 + 1);
-                    a[0] *= g0.x; a[1] *= g0.y; a[2] *= g0.z; a[3] *= g0.w;
-                    a[4] *= g1.x; a[5] *= g1.y; a[6] *= g1.z; a[7] *= g1.w;
-                } else {
-#pragma unroll
-                    for (int t = 0; t < 8; ++t) a[t] = gelu_tanh_fast(a[t]);
-                }
-                uint32_t hw[4], lw[4];
-#pragma unroll
-                for (int t = 0; t < 4; ++t) {
-                    const __nv_bfloat16 h0 = __float2bfloat16_rn(a[2 * t]), h1 = __float2bfloat16_rn(a[2 * t + 1]);
-                    const __nv_bfloat16 l0 = __float2bfloat16_rn(a[2 * t] - __bfloat162float(h0)), l1 = __float2bfloat16_rn(a[2 * t + 1] - __bfloat162float(h1));
-                    hw[t] = (uint32_t)__bfloat16_as_ushort(h0) | ((uint32_t)__bfloat16_as_ushort(h1) << 16);
-                    lw[t] = (uint32_t)__bfloat16_as_ushort(l0) | ((uint32_t)__bfloat16_as_ushort(l1) << 16);
-                }
-                // row i of the operand: 128 bytes, its 16-byte chunk c stored at position c ^ (i mod 8)
-                uint8_t *dst = smem + (size_t)j * stage_bytes + A_BYTES + i * (TILE_K * 2) + ((c ^ (i & 7)) << 4);
-                *reinterpret_cast<uint4 *>(dst) = make_uint4(hw[0], hw[1], hw[2], hw[3]);
-                if (p.use_lo) *reinterpret_cast<uint4 *>(dst + b_bytes) = make_uint4(lw[0], lw[1], lw[2], lw[3]);
-            }
-        }
-        ptx::fence_proxy_async_smem(); // the tensor core reads these stages through the asynchronous proxy
-        __syncwarp();
-        const int done = min(nu, (base + 128 * STAGE_BATCH) / cpu);
-        if (lane == 0)
-            for (int j = signalled; j < done; ++j) ptx::mbar_arrive(&bars->full[j]);
-        signalled = done;
-    }
-    if (stats) {
-        epi_sync();
-        for (int i = et; i < p.n; i += 128) {
-            atomicAdd(p.f.stats_out + 2 * i, bars->sum1[i]);
-            atomicAdd(p.f.stats_out + 2 * i + 1, bars->sum2[i]);
-        }
-        __threadfence();
-        epi_sync();
-        if (et == 0) atomicAdd(p.f.stats_counter, 1);
-    }
-}
-
-// FUSED = false is the plain projection (no fold, tail, self-staged operand or buffer clearing): it needs few enough
-// registers for three CTAs of it, or two next to the element-wise kernels' CTAs, to be resident on an SM.
-template <bool FUSED>
-__global__ void __launch_bounds__(GEMM_THREADS, FUSED ? 1 : 3)
+// (Few enough registers for three CTAs of it, or two next to the element-wise kernels' CTAs, to be resident on an SM.)
+__global__ void __launch_bounds__(GEMM_THREADS, 3)
 gemm_ws_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant__ CUtensorMap map_hi,
                const __grid_constant__ CUtensorMap map_lo, const GemmParams p) {
     extern __shared__ uint8_t smem_raw[];
@@ -218,13 +113,11 @@ gemm_ws_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant_
     ptx::pdl_launch_dependents(); // the next kernel may start: its CTAs begin their own weight prefetch as SMs have room
     if (threadIdx.x == 0) {
         ptx::trace_mark(p.trace, 0);
-        // a stage is full once its weight tile has landed and, if the CTA converts the activations itself, each of the four staging warps has arrived
-        for (int s = 0; s < p.stages; ++s) { ptx::mbar_init(&bars->full[s], (FUSED && p.f.src_mode) ? 5 : 1); ptx::mbar_init(&bars->empty[s], 1); }
+        for (int s = 0; s < p.stages; ++s) { ptx::mbar_init(&bars->full[s], 1); ptx::mbar_init(&bars->empty[s], 1); }
         for (int a = 0; a < 2; ++a) { ptx::mbar_init(&bars->acc_full[a], 1); ptx::mbar_init(&bars->acc_empty[a], 4); }
         // a device error recorded by an earlier kernel makes every later one a no-op, so that a
         // failure costs one time-out, not one per launch
         bars->abort = (*reinterpret_cast<volatile int32_t *>(p.status) != 0) ? 1u : 0u;
-        if (FUSED && p.f.src_mode && u1 - u0 > p.stages) { atomicExch(p.status, 0x600); bars->abort = 1u; } // self-staged operands need a stage per unit
         ptx::fence_mbar_init();
         // Phase 1 of the producer, issued here by the same thread: weights only, for as many units as there are stages.
         // They depend neither on the previous kernel nor on this CTA's tensor memory, whose allocation (below) waits
@@ -232,7 +125,7 @@ gemm_ws_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant_
         if (!bars->abort && u1 > u0) {
             ptx::prefetch_tensormap(&map_w);
             const uint64_t pol = ptx::policy_evict_first();
-            const uint32_t tx = (uint32_t)((FUSED && p.f.src_mode) ? A_BYTES : stage_bytes);
+            const uint32_t tx = (uint32_t)stage_bytes;
             int tile = u0 / p.k_tiles, kt = u0 - tile * p.k_tiles;
             const int pre = min(u1 - u0, p.stages);
             for (int j = 0; j < pre; ++j) {
@@ -260,8 +153,7 @@ gemm_ws_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant_
             ptx::prefetch_tensormap(&map_hi);
             if (p.use_lo) ptx::prefetch_tensormap(&map_lo);
             const uint64_t pol = ptx::policy_evict_first();
-            const bool self_staged = FUSED && p.f.src_mode;
-            const uint32_t tx = (uint32_t)(self_staged ? A_BYTES : stage_bytes);
+            const uint32_t tx = (uint32_t)stage_bytes;
             // (phase 1, the weight tiles of the first `pre` units, was issued before the CTA-wide set-up barrier)
             const int pre = min(u1 - u0, p.stages);
             // (one integer division per role, none per unit: for one thread a division is ~150 cycles, and several per unit
@@ -270,7 +162,7 @@ gemm_ws_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant_
             ptx::pdl_grid_wait(); // activations are produced by the previous kernel
             ptx::trace_mark(p.trace, 1);
             bool ok = true;
-            for (int u = u0; u < u1 && ok && !self_staged; ++u) { // (self-staged operands: every unit has a stage of its own, nothing left to load)
+            for (int u = u0; u < u1 && ok; ++u) {
                 const int j = u - u0;
                 uint8_t *st = smem + (size_t)s * stage_bytes;
                 if (j >= pre) {
@@ -331,37 +223,6 @@ gemm_ws_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant_
         ptx::pdl_grid_wait();         // Y may still be read or written by the previous kernels
         float *const y = p.y ? p.y : p.info->logits;
         const int et = threadIdx.x - 64; // 0..127 among the epilogue threads
-        if constexpr (FUSED) {
-        if (p.f.src_mode) stage_operand(p, bars, smem, stage_bytes, b_bytes, u0, u1, et, lane);
-        if (p.f.clear) { // this CTA's share of an accumulator buffer that the kernels before this one have finished with
-            float4 *c4 = reinterpret_cast<float4 *>(p.f.clear);
-            const size_t count = p.f.clear_floats / 4;
-            for (size_t e = (size_t)blockIdx.x * 128 + et; e < count; e += (size_t)gridDim.x * 128) c4[e] = make_float4(0.f, 0.f, 0.f, 0.f);
-        }
-        if (p.f.fold && p.f.stats_counter) {
-            // the statistics are complete once every CTA that holds a unit of output tile 0 has counted itself
-            if (et == 0) {
-                const unsigned units_all = (unsigned)p.n_tiles * (unsigned)p.k_tiles;
-                const int target = (int)(((unsigned)p.k_tiles * gridDim.x - 1u) / units_all) + 1;
-                const long long t0 = clock64();
-                while (*reinterpret_cast<volatile int *>(p.f.stats_counter) < target) {
-                    if (clock64() - t0 > 500000000ll) { fail(p, bars, 0x500); break; }
-                    __nanosleep(64);
-                }
-                __threadfence();
-            }
-            epi_sync();
-        }
-        if (p.f.fold || p.f.tail == TAIL_GELU_PLANES) { // statistics of the LayerNorm in front of this projection
-            for (int i = et; i < p.n; i += 128) {
-                const float2 st = __ldcg(reinterpret_cast<const float2 *>(p.f.stats_in + 2 * i));
-                const float mean = st.x * p.f.inv_d;
-                bars->mean[i] = mean;
-                bars->rstd[i] = rsqrtf(fmaxf(st.y * p.f.inv_d - mean * mean, 0.f) + p.f.eps);
-            }
-            epi_sync();
-        }
-        } // FUSED
         int seg = 0;
         bool ok = true;
         for (int u = u0; u < u1;) { // (no early exit: the four warps must meet at the same barriers)
@@ -372,8 +233,6 @@ gemm_ws_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant_
             // (what does not depend on the accumulator is fetched before waiting for it)
             const int o = tile * TILE_M + quarter * 32 + lane;
             const float bias = (has_k0 && p.bias && o < p.out) ? p.bias[o] : 0.f;
-            const bool fold = FUSED && p.f.fold;
-            const float f1 = (fold && has_k0 && o < p.out) ? p.f.c1[o] : 0.f, f2 = (fold && has_k0 && o < p.out) ? p.f.c2[o] : 0.f;
             const uint32_t taddr = tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(ab * acc_cols);
             // one lane per warp polls (spinning threads would compete with the tensor cores for shared memory)
             int good = ok ? 1 : 0;
@@ -389,7 +248,7 @@ gemm_ws_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant_
                 ptx::tmem_ld_wait();
                 if (o < p.out) {
                     float *yo = y + (size_t)c0 * p.ldy + o;
-                    if (!fold && stacked && c0 + 16 <= p.n) { // the usual case, kept short: sixteen full rows, hi + lo columns
+                    if (stacked && c0 + 16 <= p.n) { // the usual case, kept short: sixteen full rows, hi + lo columns
 #pragma unroll
                         for (int t = 0; t < 16; ++t, yo += p.ldy) ptx::red_add_f32(yo, __uint_as_float(r[t]) + __uint_as_float(q[t]) + bias);
                     } else {
@@ -398,7 +257,6 @@ gemm_ws_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant_
                             const int i = c0 + t;
                             if (i < p.n) {
                                 float v = __uint_as_float(r[t]) + (stacked ? __uint_as_float(q[t]) : 0.f) + bias;
-                                if (fold) v = bars->rstd[i] * (v - bars->mean[i] * f1) + f2;
                                 ptx::red_add_f32(yo + (size_t)t * p.ldy, v);
                             }
                         }
@@ -408,89 +266,6 @@ gemm_ws_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant_
             ptx::tc_fence_before_sync();
             __syncwarp();
             if (lane == 0) ptx::mbar_arrive(&bars->acc_empty[ab]);
-            if (FUSED && p.f.tail != TAIL_NONE) {
-                // Whoever adds the last partial sum of this output tile finishes it (the classic
-                // fence + counter pattern): partial sums are fenced, then one thread counts the arrival.
-                __threadfence();
-                epi_sync();
-                if (et == 0) {
-                    const unsigned units_all = (unsigned)p.n_tiles * (unsigned)p.k_tiles, G = gridDim.x;
-                    // CTA that owns unit u: floor(((u + 1) * G - 1) / units)
-                    const unsigned first = (((unsigned)(tile * p.k_tiles) + 1u) * G - 1u) / units_all;
-                    const unsigned last = (((unsigned)(tile * p.k_tiles + p.k_tiles - 1) + 1u) * G - 1u) / units_all;
-                    bars->tail_last = 0;
-                    if (!bars->abort) { // a CTA that gave up on a wait does not count: the tile then stays unfinished and the error word says why
-                        const int arrived = atomicAdd(p.f.tile_count + tile, 1) + 1;
-                        bars->tail_last = (arrived == (int)(last - first + 1u));
-                        if (bars->tail_last) p.f.tile_count[tile] = 0; // at rest again for the next launch
-                    }
-                }
-                epi_sync();
-                if (bars->tail_last) {
-                    __threadfence();
-                    const bool col_ok = o < p.out;
-                    if (p.f.tail == TAIL_LN_PLANES) {
-                        const float g = col_ok ? p.f.gain[o] : 0.f;
-                        for (int i0 = 0; i0 < p.n; i0 += 16) { // sixteen rows at a time: their loads fly together
-                            float v[16];
-#pragma unroll
-                            for (int q = 0; q < 16; ++q) v[q] = (col_ok && i0 + q < p.n) ? __ldcg(y + (size_t)(i0 + q) * p.ldy + o) : 0.f;
-#pragma unroll
-                            for (int q0 = 0; q0 < 16; q0 += 4) { // four independent reduction chains at a time
-                                float s1[4], s2[4];
-#pragma unroll
-                                for (int q4 = 0; q4 < 4; ++q4) { s1[q4] = v[q0 + q4]; s2[q4] = v[q0 + q4] * v[q0 + q4]; }
-#pragma unroll
-                                for (int off = 16; off > 0; off >>= 1)
-#pragma unroll
-                                    for (int q4 = 0; q4 < 4; ++q4) {
-                                        s1[q4] += __shfl_xor_sync(0xffffffffu, s1[q4], off);
-                                        s2[q4] += __shfl_xor_sync(0xffffffffu, s2[q4], off);
-                                    }
-#pragma unroll
-                                for (int q4 = 0; q4 < 4; ++q4) {
-                                    const int i = i0 + q0 + q4;
-                                    if (i < p.n) {
-                                        if (lane == 0) { atomicAdd(p.f.stats_out + 2 * i, s1[q4]); atomicAdd(p.f.stats_out + 2 * i + 1, s2[q4]); }
-                                        if (col_ok) {
-                                            const float a = v[q0 + q4] * g;
-                                            const __nv_bfloat16 h = __float2bfloat16_rn(a);
-                                            p.f.plane_hi[(size_t)i * p.f.plane_ld + o] = h;
-                                            if (p.f.plane_lo) p.f.plane_lo[(size_t)i * p.f.plane_ld + o] = __float2bfloat16_rn(a - __bfloat162float(h));
-                                        }
-                                    }
-                                }
-                            }
-                        }
-                        if (p.f.zero) { // this tile's share of the accumulators to clear
-                            const int per = (p.f.zero_cols + p.n_tiles - 1) / p.n_tiles, c0 = tile * per, c1 = min(p.f.zero_cols, c0 + per);
-                            for (int i = 0; i < p.n; ++i)
-                                for (int c = c0 + et; c < c1; c += 128) p.f.zero[(size_t)i * p.f.zero_cols + c] = 0.f;
-                        }
-                    } else { // TAIL_GELU_PLANES
-                        const float k1 = col_ok ? p.f.c1[o] : 0.f, k2 = col_ok ? p.f.c2[o] : 0.f;
-                        if (col_ok) {
-                            for (int i0 = 0; i0 < p.n; i0 += 16) {
-                                float v[16];
-#pragma unroll
-                                for (int q = 0; q < 16; ++q) v[q] = (i0 + q < p.n) ? __ldcg(y + (size_t)(i0 + q) * p.ldy + o) : 0.f;
-#pragma unroll
-                                for (int q = 0; q < 16; ++q) {
-                                    const int i = i0 + q;
-                                    if (i < p.n) {
-                                        const float a = gelu_tanh_fast(bars->rstd[i] * (v[q] - bars->mean[i] * k1) + k2);
-                                        y[(size_t)i * p.ldy + o] = 0.f; // the accumulators start the next layer at zero
-                                        const __nv_bfloat16 h = __float2bfloat16_rn(a);
-                                        p.f.plane_hi[(size_t)i * p.f.plane_ld + o] = h;
-                                        if (p.f.plane_lo) p.f.plane_lo[(size_t)i * p.f.plane_ld + o] = __float2bfloat16_rn(a - __bfloat162float(h));
-                                    }
-                                }
-                            }
-                        }
-                    }
-                }
-                epi_sync(); // tail_last is reused by the next segment
-            }
             ++seg;
             u = seg_end;
         }
@@ -544,37 +319,26 @@ int gemm_ws_stages(int n_pad, int use_lo, bool shared_sm) {
     return s > MAX_STAGES ? MAX_STAGES : (s < 2 ? 2 : s);
 }
 
-bool gemm_ws_can_self_stage(int n, int K, int out, int use_lo, int grid, int sm_count) {
-    const int n_pad = (n + 15) & ~15;
-    const long long units = (long long)((out + TILE_M - 1) / TILE_M) * (K / TILE_K);
-    if (grid > units) grid = (int)units;
-    return (units + grid - 1) / grid <= gemm_ws_stages(n_pad, use_lo, grid > sm_count);
-}
-
 cudaError_t gemm_ws_prepare() {
-    cudaError_t e = cudaFuncSetAttribute(gemm_ws_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024);
-    if (e == cudaSuccess) e = cudaFuncSetAttribute(gemm_ws_kernel<false>, cudaFuncAttributePreferredSharedMemoryCarveout, cudaSharedmemCarveoutMaxShared);
-    if (e == cudaSuccess) e = cudaFuncSetAttribute(gemm_ws_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024);
-    if (e == cudaSuccess) e = cudaFuncSetAttribute(gemm_ws_kernel<true>, cudaFuncAttributePreferredSharedMemoryCarveout, cudaSharedmemCarveoutMaxShared);
+    cudaError_t e = cudaFuncSetAttribute(gemm_ws_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024);
+    if (e == cudaSuccess) e = cudaFuncSetAttribute(gemm_ws_kernel, cudaFuncAttributePreferredSharedMemoryCarveout, cudaSharedmemCarveoutMaxShared);
     return e;
 }
 
 cudaError_t launch_gemm_ws(const void *map_w, const void *map_hi, const void *map_lo, float *y, const StepInfo *info, int ldy,
                            const float *bias, int n, int K, int out, int use_lo, int grid, int sm_count, int32_t *status, bool pdl,
-                           cudaStream_t s, const GemmFusion *fusion, unsigned long long *trace) {
+                           cudaStream_t s, unsigned long long *trace) {
     GemmParams p;
     p.trace = trace;
-    if (fusion) p.f = *fusion; else memset(&p.f, 0, sizeof(p.f));
     p.y = y; p.info = info; p.bias = bias; p.n = n; p.n_pad = (n + 15) & ~15;
     p.out = out; p.ldy = ldy; p.k_tiles = K / TILE_K; p.n_tiles = (out + TILE_M - 1) / TILE_M;
     p.use_lo = use_lo; p.status = status;
-    const bool fused = p.f.fold || p.f.tail != TAIL_NONE || p.f.src_mode != SRC_TMA || p.f.clear;
     const int stage_bytes = A_BYTES + p.n_pad * TILE_K * 2 * (use_lo ? 2 : 1);
     const long long units = (long long)p.n_tiles * p.k_tiles;
     if (grid > units) grid = (int)units;
     int per_cta = (int)((units + grid - 1) / grid);
     p.split = 0;
-    if (!fused && grid >= p.n_tiles) {
+    if (grid >= p.n_tiles) {
         // When there are at least as many CTAs as output tiles, give every tile its own group of CTAs: a CTA whose range
         // straddles two tiles runs two epilogues, and the kernel ends with its slowest CTA.
         int most = grid / p.n_tiles;
@@ -587,9 +351,11 @@ cudaError_t launch_gemm_ws(const void *map_w, const void *map_hi, const void *ma
         grid = p.split * p.n_tiles;
     }
     p.stages = gemm_ws_stages(p.n_pad, use_lo, grid > sm_count);
-    if (p.f.src_mode && per_cta > p.stages) return cudaErrorInvalidValue; // see gemm_ws_can_self_stage
     if (p.stages > per_cta) p.stages = per_cta < 1 ? 1 : per_cta;
-    const size_t smem = (size_t)p.stages * stage_bytes + sizeof(Barriers) + 1024;
+    size_t smem = (size_t)p.stages * stage_bytes + sizeof(Barriers) + 1024;
+    // Two CTAs per SM, not three: with a third one resident the slowest CTA of a projection ends later (measured: 1.19 ms per
+    // GPT-2-large verification of 32 nodes against 1.09 ms), so a CTA asks for more than a third of an SM's shared memory.
+    if (grid > sm_count && smem < 78 * 1024) smem = 78 * 1024;
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3(grid);
     cfg.blockDim = dim3(GEMM_THREADS);
@@ -600,6 +366,6 @@ cudaError_t launch_gemm_ws(const void *map_w, const void *map_hi, const void *ma
     attr[0].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attr;
     cfg.numAttrs = pdl ? 1 : 0;
-    return cudaLaunchKernelEx(&cfg, fused ? gemm_ws_kernel<true> : gemm_ws_kernel<false>, *(const CUtensorMap *)map_w,
+    return cudaLaunchKernelEx(&cfg, gemm_ws_kernel, *(const CUtensorMap *)map_w,
                               *(const CUtensorMap *)map_hi, *(const CUtensorMap *)(map_lo ? map_lo : map_hi), p);
 }

@@ -130,6 +130,23 @@ __global__ void __launch_bounds__(256) gelu_prep_kernel(const float *__restrict_
     if (trace) { __syncthreads(); if (threadIdx.x == 0) ptx::trace_mark(trace, 2); }
 }
 
+// c1[o] = sum_k g[k] W[o,k] ; c2[o] = sum_k beta[k] W[o,k] + bias[o]   (one warp per output feature; load time only)
+__global__ void ln_fold_kernel(const __nv_bfloat16 *__restrict__ W, const float *__restrict__ g, const float *__restrict__ beta,
+                               const float *__restrict__ bias, int out, int K, float *__restrict__ c1, float *__restrict__ c2) {
+    const int o = (blockIdx.x * blockDim.x + threadIdx.x) >> 5, lane = threadIdx.x & 31;
+    if (o >= out) return;
+    const __nv_bfloat16 *w = W + (size_t)o * K;
+    float a = 0.f, b = 0.f;
+    for (int k = lane; k < K; k += 32) {
+        const float wv = __bfloat162float(w[k]);
+        a = fmaf(g[k], wv, a);
+        b = fmaf(beta[k], wv, b);
+    }
+#pragma unroll
+    for (int off = 16; off > 0; off >>= 1) { a += __shfl_xor_sync(0xffffffffu, a, off); b += __shfl_xor_sync(0xffffffffu, b, off); }
+    if (lane == 0) { c1[o] = a; c2[o] = b + (bias ? bias[o] : 0.f); }
+}
+
 template <typename... Args>
 cudaError_t launch_pdl(void (*kernel)(Args...), dim3 grid, dim3 block, cudaStream_t s, bool pdl, Args... args) {
     cudaLaunchConfig_t cfg = {};
@@ -152,6 +169,12 @@ cudaError_t prep_kernels_prepare() {
     if (e == cudaSuccess) e = cudaFuncSetAttribute(ln_prep_kernel<8>, cudaFuncAttributePreferredSharedMemoryCarveout, cudaSharedmemCarveoutMaxShared);
     if (e == cudaSuccess) e = cudaFuncSetAttribute(gelu_prep_kernel, cudaFuncAttributePreferredSharedMemoryCarveout, cudaSharedmemCarveoutMaxShared);
     return e;
+}
+
+cudaError_t launch_ln_fold(const void *W, const float *g, const float *beta, const float *bias, int out, int K, float *c1, float *c2, cudaStream_t s) {
+    const int threads = 256, warps_per_block = threads / 32;
+    ln_fold_kernel<<<(out + warps_per_block - 1) / warps_per_block, threads, 0, s>>>((const __nv_bfloat16 *)W, g, beta, bias, out, K, c1, c2);
+    return cudaGetLastError();
 }
 
 cudaError_t launch_ln_prep(const float *x, const float *g, const float *b, int n, int d, float eps, __nv_bfloat16 *a_hi, __nv_bfloat16 *a_lo,

@@ -84,15 +84,13 @@ __global__ void embed_kernel(const WT *__restrict__ wte, const WT *__restrict__ 
     for (int k = threadIdx.x; k < d; k += blockDim.x) x[(size_t)i * d + k] = (float)te[k] + (float)pe[k];
 }
 
-// Embedding for the LayerNorm-folded tensor-core path.  Besides x it writes, per row, the bf16 hi/lo
-// planes of x * gain (operand of the first QKV projection) and the row's sum / sum of squares (statistics
-// of the first LayerNorm), and it clears what the step accumulates into: the other layers' statistics and
-// the QKV / FC accumulators.
-__global__ void __launch_bounds__(256) embed_fold_kernel(const __nv_bfloat16 *__restrict__ wte, const __nv_bfloat16 *__restrict__ wpe, TreeMeta m,
-                                                         int d, const float *__restrict__ gain, float *__restrict__ x,
-                                                         __nv_bfloat16 *__restrict__ plane_hi, __nv_bfloat16 *__restrict__ plane_lo,
-                                                         float *__restrict__ stats, int stats_floats, float *__restrict__ qkv, int qkv_cols,
-                                                         float *__restrict__ fc, int fc_cols) {
+// Embedding for the cluster-reduced tensor-core path: x, the bf16 hi/lo planes of x * gain (operand of the first
+// QKV projection, whose LayerNorm is folded into its epilogue) and the row's (sum, sum of squares) as part 0 of the
+// statistics.  One CTA per row.
+__global__ void __launch_bounds__(256) embed_planes_kernel(const __nv_bfloat16 *__restrict__ wte, const __nv_bfloat16 *__restrict__ wpe, TreeMeta m,
+                                                           int d, const float *__restrict__ gain, float *__restrict__ x,
+                                                           __nv_bfloat16 *__restrict__ plane_hi, __nv_bfloat16 *__restrict__ plane_lo,
+                                                           float *__restrict__ stats) {
     __shared__ float red[8];
     const int i = blockIdx.x;
     const __nv_bfloat16 *te = wte + (size_t)m.tokens[i] * d;
@@ -110,41 +108,28 @@ __global__ void __launch_bounds__(256) embed_fold_kernel(const __nv_bfloat16 *__
     }
     s1 = block_sum_256(s1, red);
     s2 = block_sum_256(s2, red);
-    // statistics: slot 0 (first LayerNorm of layer 0) is set here, every other slot starts the step at zero
-    const int slot_floats = 2 * SSD_MAX_NODES;
-    for (int e = blockIdx.x * 256 + threadIdx.x; e < stats_floats; e += gridDim.x * 256)
-        if (e >= slot_floats) stats[e] = 0.f;
     if (threadIdx.x == 0) { stats[2 * i] = s1; stats[2 * i + 1] = s2; }
-    for (int k = threadIdx.x; k < qkv_cols; k += 256) qkv[(size_t)i * qkv_cols + k] = 0.f;
-    for (int k = threadIdx.x; k < fc_cols; k += 256) fc[(size_t)i * fc_cols + k] = 0.f;
 }
 
-cudaError_t launch_embed_fold(const void *wte, const void *wpe, const TreeMeta &m, int n, int d, const float *gain, float *x, void *plane_hi,
-                              void *plane_lo, float *stats, int stats_floats, float *qkv, int qkv_cols, float *fc, int fc_cols,
-                              cudaStream_t s) {
-    embed_fold_kernel<<<n, 256, 0, s>>>((const __nv_bfloat16 *)wte, (const __nv_bfloat16 *)wpe, m, d, gain, x, (__nv_bfloat16 *)plane_hi,
-                                        (__nv_bfloat16 *)plane_lo, stats, stats_floats, qkv, qkv_cols, fc, fc_cols);
+cudaError_t launch_embed_planes(const void *wte, const void *wpe, const TreeMeta &m, int n, int d, const float *gain, float *x, void *plane_hi,
+                                void *plane_lo, float *stats, cudaStream_t s) {
+    embed_planes_kernel<<<n, 256, 0, s>>>((const __nv_bfloat16 *)wte, (const __nv_bfloat16 *)wpe, m, d, gain, x, (__nv_bfloat16 *)plane_hi,
+                                          (__nv_bfloat16 *)plane_lo, stats);
     return cudaGetLastError();
 }
 
-// logits[n, V] = 0 (the LM-head projection accumulates its stream-K partial sums into them)
-__global__ void zero_logits_kernel(const StepInfo *__restrict__ info, size_t count) {
-    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
-    asm volatile("griddepcontrol.wait;" ::: "memory");
-    float *dst = info->logits;
-    for (size_t e = (size_t)blockIdx.x * blockDim.x + threadIdx.x; e < count; e += (size_t)gridDim.x * blockDim.x) dst[e] = 0.f;
+// logits[n, V] = 0 (the LM-head projection adds its stream-K partial sums into them).  Launched at the start of a
+// forward, as wide as the GPU, so that the clearing is off the path between the last layer and the LM head.
+__global__ void __launch_bounds__(256) zero_logits_kernel(const StepInfo *__restrict__ info, size_t count) {
+    float *dst = info->logits; // (written by the tree-preparation kernel, which precedes this one in the stream)
+    const size_t stride = (size_t)gridDim.x * blockDim.x, count4 = (reinterpret_cast<uintptr_t>(dst) & 15) == 0 ? count / 4 : 0;
+    float4 *d4 = reinterpret_cast<float4 *>(dst);
+    for (size_t e = (size_t)blockIdx.x * blockDim.x + threadIdx.x; e < count4; e += stride) d4[e] = make_float4(0.f, 0.f, 0.f, 0.f);
+    for (size_t e = 4 * count4 + (size_t)blockIdx.x * blockDim.x + threadIdx.x; e < count; e += stride) dst[e] = 0.f;
 }
-cudaError_t launch_zero_logits(const StepInfo *info, int n, int vocab, bool pdl, cudaStream_t s) {
-    cudaLaunchConfig_t cfg = {};
-    cfg.gridDim = dim3(148 * 2);
-    cfg.blockDim = dim3(256);
-    cfg.stream = s;
-    cudaLaunchAttribute attr[1];
-    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
-    attr[0].val.programmaticStreamSerializationAllowed = 1;
-    cfg.attrs = attr;
-    cfg.numAttrs = pdl ? 1 : 0;
-    return cudaLaunchKernelEx(&cfg, zero_logits_kernel, info, (size_t)n * vocab);
+cudaError_t launch_zero_logits(const StepInfo *info, int n, int vocab, cudaStream_t s) {
+    zero_logits_kernel<<<148 * 4, 256, 0, s>>>(info, (size_t)n * vocab);
+    return cudaGetLastError();
 }
 
 cudaError_t launch_embed(const void *wte, const void *wpe, int dtype, const TreeMeta &m, int n, int d, float *x, cudaStream_t s) {

@@ -6,7 +6,6 @@
 #include <new>
 #include <vector>
 
-#include "k_mega.h"
 #include "ssd_internal.h"
 
 struct ssd_kv {
@@ -43,19 +42,13 @@ struct ssd_ctx {
     TensorMap map_wte;
     std::vector<TensorMap> map_layers; // 4 per layer: qkv, o, fc, proj
     bool tensor_path;                  // bf16 model: projections on tcgen05
-    int use_lo, pdl, gemm_grid, head_grid, trace_kernels, trace_count, use_graph, use_mega, use_fused, use_staged;
-    // LayerNorm-folded per-kernel path: folded vectors (host copy of the per-layer table, LM head), row
-    // statistics [(2L + 1) slots][256 rows][2], arrival counters of the fused tails
-    std::vector<mega::LayerVecs> h_vecs;
-    float *c1_head, *c2_head, *d_fstats;
-    int32_t *d_tile_count;
-    // persistent forward kernel (trees of up to 64 nodes)
-    CUtensorMap *d_maps;      // device copies of map_layers
-    mega::LayerVecs *d_vecs;
-    float *d_stats;
-    uint32_t *d_stats_count, *d_ctrl; // ctrl[0] grid barrier, ctrl[1] abort flag
+    int use_lo, pdl, gemm_grid, head_grid, trace_kernels, trace_count, use_graph, use_cluster, cl_max, cl_size[4], attn_lo;
+    // cluster-reduced path: per-layer vectors that fold a LayerNorm into the projection behind it (c1 = W gain,
+    // c2 = W beta + bias), and the two row-statistics buffers [tile][SSD_MAX_NODES][2] (in front of QKV / of FC)
+    struct LayerFold { float *c1_qkv, *c2_qkv, *c1_fc, *c2_fc; };
+    std::vector<LayerFold> folds;
+    float *d_stats1, *d_stats2;
     unsigned long long *d_trace;
-    float *d_att_part_o, *d_att_part_ml;
     int sm_count;
     StepInfo *d_info;                  // device copy of the current step's values
     // One captured forward per tree size: the kernels read everything that changes from step to
@@ -156,8 +149,7 @@ int upload_vector_f32(ssd_ctx *ctx, const void *src, size_t count, const float *
     return SSD_OK;
 }
 
-static const ssd_ctx::ActMaps *act_maps_for(ssd_ctx *ctx, int n) {
-    const int n_pad = (n + 15) & ~15;
+static const ssd_ctx::ActMaps *act_maps_pad(ssd_ctx *ctx, int n_pad) {
     ssd_ctx::ActMaps &am = ctx->act_maps[n_pad / 16 - 1];
     if (!am.built) {
         const size_t d = ctx->cfg.d_model, F = ctx->cfg.d_ff, rows = ctx->plane_rows;
@@ -173,6 +165,8 @@ static const ssd_ctx::ActMaps *act_maps_for(ssd_ctx *ctx, int n) {
     return &am;
 }
 
+static const ssd_ctx::ActMaps *act_maps_for(ssd_ctx *ctx, int n) { return act_maps_pad(ctx, (n + 15) & ~15); }
+
 // CTAs per projection kernel.  Unless set by hand: two per SM while the tree is small enough for two CTAs' pipelines
 // and accumulators to share an SM (measured: 1.63 ms against 1.88 ms per GPT-2-large verification of 32 nodes), else one.
 static int gemm_grid_for(const ssd_ctx *ctx, int n) {
@@ -180,6 +174,11 @@ static int gemm_grid_for(const ssd_ctx *ctx, int n) {
     return ((n + 15) & ~15) <= 64 ? 2 * ctx->sm_count : ctx->sm_count;
 }
 static int head_grid_for(const ssd_ctx *ctx, int n) { return ctx->head_grid > 0 ? ctx->head_grid : gemm_grid_for(ctx, n); }
+
+// Timeline slots of the next launch (profiling aid, off by default).
+static unsigned long long *trace_slot(ssd_ctx *ctx, int kernels) {
+    return (ctx->trace_kernels && 8 * (kernels + 1) <= SSD_TRACE_SLOTS) ? ctx->d_trace + 8 * (size_t)kernels : nullptr;
+}
 
 // Enqueue every kernel of one tree-batched forward on `s`.
 cudaError_t enqueue_forward(ssd_ctx *ctx, int n, int cap, const NodeList &tk, const NodeList &pr, const StepInfo &step, cudaStream_t s,
@@ -193,112 +192,77 @@ cudaError_t enqueue_forward(ssd_ctx *ctx, int n, int cap, const NodeList &tk, co
     cudaError_t e;
 #define Q(call) do { if ((e = (call)) != cudaSuccess) return e; ++*kernels; } while (0)
     Q(launch_tree_prep(tk, pr, step, ctx->meta, ctx->d_info, s));
-    if (ctx->tensor_path && ctx->use_staged && !ctx->use_fused && gemm_ws_can_self_stage(n, c.d_model, 3 * c.d_model, ctx->use_lo, gemm_grid_for(ctx, n), ctx->sm_count) &&
-        gemm_ws_can_self_stage(n, c.d_model, c.d_ff, ctx->use_lo, gemm_grid_for(ctx, n), ctx->sm_count) &&
-        gemm_ws_can_self_stage(n, c.d_ff, c.d_model, ctx->use_lo, gemm_grid_for(ctx, n), ctx->sm_count)) {
-        // Five launches per layer and no preparation kernels: the projections that follow a LayerNorm or the
-        // GELU convert their activations themselves.  A LayerNorm is folded: the projection runs on x * gain and
-        // whoever consumes its accumulators (the attention kernel, the FC epilogue) applies mean, rstd and the
-        // precomputed vectors c1 = W gain, c2 = W beta + bias.
+    if (ctx->tensor_path) Q(launch_zero_logits(info, n, c.vocab, s)); // the LM head adds its stream-K partial sums into them
+    if (ctx->tensor_path && ctx->use_cluster && gemm_cl_supports(n, c.d_model)) {
+        // bf16 model, trees of up to 64 nodes: five launches per layer.  Every projection reduces its split-K partial sums
+        // inside a thread-block cluster, so its epilogue holds finished sums and does the work that would otherwise be
+        // kernels of their own: the LayerNorms are folded (the projection runs on x * gain; mean, rstd and the precomputed
+        // c1 = W gain, c2 = W beta + bias are applied to the sums), GELU is applied where the FC sums are complete, and the
+        // residual additions write the next operand planes and the next LayerNorm's row statistics.
         const bool pdl = ctx->pdl != 0;
-        const int lo = ctx->use_lo, grid = gemm_grid_for(ctx, n), slot = 2 * SSD_MAX_NODES, L = c.n_layer;
-        __nv_bfloat16 *a_lo = lo ? ctx->a_lo : nullptr, *o_lo = lo ? ctx->o_lo : nullptr;
-        auto T = [&]() -> unsigned long long * { // timeline slots of the next launch (profiling aid, off by default)
-            return (ctx->trace_kernels && 8 * (*kernels + 1) <= mega::TRACE_SLOTS) ? ctx->d_trace + 8 * (size_t)*kernels : nullptr;
+        const int lo = ctx->use_lo, sms = ctx->sm_count, L = c.n_layer, n_pad = gemm_cl_n_pad(n);
+        const bool two = n_pad <= 32; // two CTAs' pipelines and reduction buffers fit one SM
+        const ssd_ctx::ActMaps *amh = am; // (the LM head's operand box is the tree's own padded size)
+        am = act_maps_pad(ctx, n_pad);
+        if (!am) return cudaErrorUnknown;
+        // (one SM's worth of CTAs per projection: the next projection's CTAs are resident beside them and prefetch their weights)
+        const int slots = ctx->gemm_grid > 0 ? ctx->gemm_grid : sms, cmax = ctx->cl_max;
+        const int tiles_d = (d + 127) / 128;
+        auto pick = [&](int which, int K, int out) { // a cluster size set by hand is still cut down to one the kernel can run
+            return ctx->cl_size[which] > 0 ? gemm_cl_cluster_size(n, K, out, 1 << 20, ctx->cl_size[which]) : gemm_cl_cluster_size(n, K, out, slots, cmax);
         };
-        int *counters = reinterpret_cast<int *>(ctx->d_fstats + (size_t)(2 * L + 1) * slot);
-        Q(launch_embed_fold(ctx->wte, ctx->wpe, ctx->meta, n, d, ctx->h_vecs[0].ln1_g, ctx->x, ctx->a_hi, a_lo, ctx->d_fstats,
-                            (2 * L + 1) * slot + (2 * L + 1), ctx->qkv, 3 * d, ctx->h, F, s));
-        for (int l = 0; l < L; ++l) {
-            const LayerWeights &Lw = ctx->layers[l];
-            const mega::LayerVecs &v = ctx->h_vecs[l];
-            const TensorMap *t = &ctx->map_layers[(size_t)4 * l];
-            float *st1 = ctx->d_fstats + (size_t)(2 * l) * slot, *st2 = st1 + slot;
-            GemmFusion fq = {};
-            fq.src_mode = SRC_LN_GAIN; fq.src = ctx->x; fq.src_ld = d; fq.gain = Lw.ln1_g;
-            fq.stats_out = l > 0 ? st1 : nullptr; // (layer 0: written by the embedding kernel)
-            fq.stats_counter = counters + 2 * l;
-            fq.clear = ctx->h; fq.clear_floats = (size_t)n * F; // FC accumulators: the previous layer's output projection has read them
-            Q(launch_gemm_ws(&t[0], &am->a_hi, &am->a_lo, ctx->qkv, info, 3 * d, nullptr, n, d, 3 * d, lo, grid, ctx->sm_count, ctx->d_status, pdl, s, &fq, T()));
-            Q(launch_tree_attention_mma(ctx->qkv, info, l * layer_elems, ctx->meta, n, c.n_head, cap, ctx->o_hi, o_lo, pdl, s, st1, v.c1_qkv, v.c2_qkv,
-                                        c.ln_eps, T()));
-            GemmFusion fo = {};
-            fo.clear = ctx->qkv; fo.clear_floats = (size_t)n * 3 * d; // the attention kernel has read them
-            Q(launch_gemm_ws(&t[1], &am->o_hi, &am->o_lo, ctx->x, info, d, Lw.b_o, n, d, d, lo, grid, ctx->sm_count, ctx->d_status, pdl, s, &fo, T()));
-            GemmFusion ff = {};
-            ff.src_mode = SRC_LN_GAIN; ff.src = ctx->x; ff.src_ld = d; ff.gain = Lw.ln2_g; ff.stats_out = st2; ff.stats_counter = counters + 2 * l + 1;
-            ff.fold = 1; ff.stats_in = st2; ff.c1 = v.c1_fc; ff.c2 = v.c2_fc; ff.inv_d = 1.0f / d; ff.eps = c.ln_eps;
-            Q(launch_gemm_ws(&t[2], &am->a_hi, &am->a_lo, ctx->h, info, F, nullptr, n, d, F, lo, grid, ctx->sm_count, ctx->d_status, pdl, s, &ff, T()));
-            GemmFusion fp = {};
-            fp.src_mode = SRC_GELU; fp.src = ctx->h; fp.src_ld = F;
-            Q(launch_gemm_ws(&t[3], &am->h_hi, &am->h_lo, ctx->x, info, d, Lw.b_proj, n, F, d, lo, grid, ctx->sm_count, ctx->d_status, pdl, s, &fp, T()));
-        }
-        Q(launch_ln_prep(ctx->x, ctx->lnf_g, ctx->lnf_b, n, d, c.ln_eps, ctx->a_hi, a_lo, nullptr, c.vocab, info, 1, pdl, s, T()));
-        Q(launch_gemm_ws(&ctx->map_wte, &am->a_hi, &am->a_lo, nullptr, info, c.vocab, nullptr, n, d, c.vocab, lo, head_grid_for(ctx, n), ctx->sm_count, ctx->d_status, pdl, s, nullptr, T()));
-        ctx->trace_count = ctx->trace_kernels ? 8 * *kernels : 0;
-        return cudaSuccess;
-    }
-    if (ctx->tensor_path && ctx->use_fused) {
-        // Five launches per layer.  The LayerNorms are folded into the projections that follow them
-        // (computed on x * gain, normalised in the consumer), and whichever CTA completes an output
-        // tile of a projection also prepares the next projection's operand planes.
-        const bool pdl = ctx->pdl != 0;
-        const int lo = ctx->use_lo, grid = gemm_grid_for(ctx, n), slot = 2 * SSD_MAX_NODES, L = c.n_layer;
+        const int s_qkv = pick(0, d, 3 * d), s_o = pick(1, d, d), s_fc = pick(2, d, F), s_proj = pick(3, F, d);
         __nv_bfloat16 *a_lo = lo ? ctx->a_lo : nullptr, *o_lo = lo ? ctx->o_lo : nullptr, *h_lo = lo ? ctx->h_lo : nullptr;
-        Q(launch_embed_fold(ctx->wte, ctx->wpe, ctx->meta, n, d, ctx->h_vecs[0].ln1_g, ctx->x, ctx->a_hi, a_lo, ctx->d_fstats, (2 * L + 1) * slot,
-                            ctx->qkv, 3 * d, ctx->h, F, s));
+        Q(launch_embed_planes(ctx->wte, ctx->wpe, ctx->meta, n, d, ctx->layers[0].ln1_g, ctx->x, ctx->a_hi, a_lo, ctx->d_stats1, s));
         for (int l = 0; l < L; ++l) {
             const LayerWeights &Lw = ctx->layers[l];
-            const mega::LayerVecs &v = ctx->h_vecs[l];
+            const ssd_ctx::LayerFold &v = ctx->folds[l];
             const TensorMap *t = &ctx->map_layers[(size_t)4 * l];
-            float *st1 = ctx->d_fstats + (size_t)(2 * l) * slot, *st2 = st1 + slot, *st_next = st2 + slot;
-            Q(launch_gemm_ws(&t[0], &am->a_hi, &am->a_lo, ctx->qkv, info, 3 * d, nullptr, n, d, 3 * d, lo, grid, ctx->sm_count, ctx->d_status, pdl, s));
-            Q(launch_tree_attention_mma(ctx->qkv, info, l * layer_elems, ctx->meta, n, c.n_head, cap, ctx->o_hi, o_lo, pdl, s, st1, v.c1_qkv, v.c2_qkv,
-                                        c.ln_eps));
-            GemmFusion fo = {};
-            fo.tail = TAIL_LN_PLANES; fo.gain = Lw.ln2_g; fo.stats_out = st2; fo.plane_hi = ctx->a_hi; fo.plane_lo = a_lo; fo.plane_ld = d;
-            fo.zero = ctx->qkv; fo.zero_cols = 3 * d; fo.tile_count = ctx->d_tile_count;
-            Q(launch_gemm_ws(&t[1], &am->o_hi, &am->o_lo, ctx->x, info, d, Lw.b_o, n, d, d, lo, grid, ctx->sm_count, ctx->d_status, pdl, s, &fo));
-            GemmFusion ff = {};
-            ff.tail = TAIL_GELU_PLANES; ff.stats_in = st2; ff.c1 = v.c1_fc; ff.c2 = v.c2_fc; ff.inv_d = 1.0f / d; ff.eps = c.ln_eps;
-            ff.plane_hi = ctx->h_hi; ff.plane_lo = h_lo; ff.plane_ld = F; ff.tile_count = ctx->d_tile_count + 256;
-            Q(launch_gemm_ws(&t[2], &am->a_hi, &am->a_lo, ctx->h, info, F, nullptr, n, d, F, lo, grid, ctx->sm_count, ctx->d_status, pdl, s, &ff));
-            GemmFusion fp = {};
-            fp.tail = TAIL_LN_PLANES; fp.gain = (l + 1 < L) ? ctx->h_vecs[l + 1].ln1_g : ctx->lnf_g; fp.stats_out = st_next;
-            fp.plane_hi = ctx->a_hi; fp.plane_lo = a_lo; fp.plane_ld = d; fp.tile_count = ctx->d_tile_count + 512;
-            Q(launch_gemm_ws(&t[3], &am->h_hi, &am->h_lo, ctx->x, info, d, Lw.b_proj, n, F, d, lo, grid, ctx->sm_count, ctx->d_status, pdl, s, &fp));
+            GemmClEpilogue eq = {};
+            eq.mode = MODE_FOLD_STORE; eq.stats_in = ctx->d_stats1; eq.stats_parts = l == 0 ? 1 : tiles_d; eq.c1 = v.c1_qkv; eq.c2 = v.c2_qkv;
+            eq.inv_d = 1.0f / d; eq.eps = c.ln_eps; eq.y = ctx->qkv; eq.ldy = 3 * d;
+            Q(launch_gemm_cl(&t[0], &am->a_hi, &am->a_lo, n, d, 3 * d, lo, s_qkv, two, eq, ctx->d_status, pdl, s, trace_slot(ctx, *kernels)));
+            Q(launch_tree_attention_mma(ctx->qkv, info, l * layer_elems, ctx->meta, n, c.n_head, cap, ctx->o_hi, o_lo, pdl, s, trace_slot(ctx, *kernels), ctx->attn_lo != 0));
+            GemmClEpilogue eo = {};
+            eo.mode = MODE_RESIDUAL; eo.y = ctx->x; eo.ldy = d; eo.bias = Lw.b_o; eo.gain = Lw.ln2_g; eo.plane_hi = ctx->a_hi; eo.plane_lo = a_lo;
+            eo.plane_ld = d; eo.stats_out = ctx->d_stats2;
+            Q(launch_gemm_cl(&t[1], &am->o_hi, &am->o_lo, n, d, d, lo, s_o, two, eo, ctx->d_status, pdl, s, trace_slot(ctx, *kernels)));
+            GemmClEpilogue ef = {};
+            ef.mode = MODE_FOLD_GELU; ef.stats_in = ctx->d_stats2; ef.stats_parts = tiles_d; ef.c1 = v.c1_fc; ef.c2 = v.c2_fc; ef.inv_d = 1.0f / d;
+            ef.eps = c.ln_eps; ef.plane_hi = ctx->h_hi; ef.plane_lo = h_lo; ef.plane_ld = F;
+            Q(launch_gemm_cl(&t[2], &am->a_hi, &am->a_lo, n, d, F, lo, s_fc, two, ef, ctx->d_status, pdl, s, trace_slot(ctx, *kernels)));
+            GemmClEpilogue ep = {};
+            ep.mode = MODE_RESIDUAL; ep.y = ctx->x; ep.ldy = d; ep.bias = Lw.b_proj; ep.gain = l + 1 < L ? ctx->layers[l + 1].ln1_g : nullptr;
+            ep.plane_hi = ctx->a_hi; ep.plane_lo = a_lo; ep.plane_ld = d; ep.stats_out = ctx->d_stats1;
+            Q(launch_gemm_cl(&t[3], &am->h_hi, &am->h_lo, n, F, d, lo, s_proj, two, ep, ctx->d_status, pdl, s, trace_slot(ctx, *kernels)));
         }
-        Q(launch_zero_logits(info, n, c.vocab, pdl, s));
-        GemmFusion fh = {};
-        fh.fold = 1; fh.stats_in = ctx->d_fstats + (size_t)(2 * L) * slot; fh.c1 = ctx->c1_head; fh.c2 = ctx->c2_head; fh.inv_d = 1.0f / d; fh.eps = c.ln_eps;
-        Q(launch_gemm_ws(&ctx->map_wte, &am->a_hi, &am->a_lo, nullptr, info, c.vocab, nullptr, n, d, c.vocab, lo, head_grid_for(ctx, n), ctx->sm_count, ctx->d_status, pdl, s, &fh));
+        const int hgrid = head_grid_for(ctx, n);
+        Q(launch_ln_prep(ctx->x, ctx->lnf_g, ctx->lnf_b, n, d, c.ln_eps, ctx->a_hi, a_lo, nullptr, 0, info, 0, pdl, s, trace_slot(ctx, *kernels)));
+        Q(launch_gemm_ws(&ctx->map_wte, &amh->a_hi, &amh->a_lo, nullptr, info, c.vocab, nullptr, n, d, c.vocab, lo, hgrid, sms, ctx->d_status, pdl, s, trace_slot(ctx, *kernels)));
+        ctx->trace_count = ctx->trace_kernels ? 8 * *kernels : 0;
         return cudaSuccess;
     }
     Q(launch_embed(ctx->wte, ctx->wpe, c.dtype, ctx->meta, n, d, ctx->x, s));
     if (ctx->tensor_path) {
-        // bf16 model: LayerNorm / GELU feed bf16 operand planes, projections run on the tensor
-        // cores and accumulate into fp32 buffers; every kernel is a programmatic dependent launch.
+        // bf16 model, the default path: LayerNorm / GELU kernels feed bf16 operand planes, projections
+        // accumulate their stream-K partial sums into fp32 buffers; every kernel is a programmatic dependent launch.
         const bool pdl = ctx->pdl != 0;
         const int lo = ctx->use_lo, grid = gemm_grid_for(ctx, n), hgrid = head_grid_for(ctx, n), sms = ctx->sm_count;
         __nv_bfloat16 *a_lo = lo ? ctx->a_lo : nullptr, *o_lo = lo ? ctx->o_lo : nullptr, *h_lo = lo ? ctx->h_lo : nullptr;
-        // timeline slots of the next launch (profiling aid, off by default)
-        auto T = [&]() -> unsigned long long * {
-            return (ctx->trace_kernels && 8 * (*kernels + 1) <= mega::TRACE_SLOTS) ? ctx->d_trace + 8 * (size_t)*kernels : nullptr;
-        };
         for (int l = 0; l < c.n_layer; ++l) {
             const LayerWeights &L = ctx->layers[l];
             const TensorMap *t = &ctx->map_layers[(size_t)4 * l];
-            Q(launch_ln_prep(ctx->x, L.ln1_g, L.ln1_b, n, d, c.ln_eps, ctx->a_hi, a_lo, ctx->qkv, 3 * d, info, 0, pdl, s, T()));
-            Q(launch_gemm_ws(&t[0], &am->a_hi, &am->a_lo, ctx->qkv, info, 3 * d, L.b_qkv, n, d, 3 * d, lo, grid, sms, ctx->d_status, pdl, s, nullptr, T()));
-            Q(launch_tree_attention_mma(ctx->qkv, info, l * layer_elems, ctx->meta, n, c.n_head, cap, ctx->o_hi, o_lo, pdl, s, nullptr, nullptr, nullptr, 0.f, T()));
-            Q(launch_gemm_ws(&t[1], &am->o_hi, &am->o_lo, ctx->x, info, d, L.b_o, n, d, d, lo, grid, sms, ctx->d_status, pdl, s, nullptr, T()));
-            Q(launch_ln_prep(ctx->x, L.ln2_g, L.ln2_b, n, d, c.ln_eps, ctx->a_hi, a_lo, ctx->h, F, info, 0, pdl, s, T()));
-            Q(launch_gemm_ws(&t[2], &am->a_hi, &am->a_lo, ctx->h, info, F, L.b_fc, n, d, F, lo, grid, sms, ctx->d_status, pdl, s, nullptr, T()));
-            Q(launch_gelu_prep(ctx->h, n, F, ctx->h_hi, h_lo, pdl, s, T()));
-            Q(launch_gemm_ws(&t[3], &am->h_hi, &am->h_lo, ctx->x, info, d, L.b_proj, n, F, d, lo, grid, sms, ctx->d_status, pdl, s, nullptr, T()));
+            Q(launch_ln_prep(ctx->x, L.ln1_g, L.ln1_b, n, d, c.ln_eps, ctx->a_hi, a_lo, ctx->qkv, 3 * d, info, 0, pdl, s, trace_slot(ctx, *kernels)));
+            Q(launch_gemm_ws(&t[0], &am->a_hi, &am->a_lo, ctx->qkv, info, 3 * d, L.b_qkv, n, d, 3 * d, lo, grid, sms, ctx->d_status, pdl, s, trace_slot(ctx, *kernels)));
+            Q(launch_tree_attention_mma(ctx->qkv, info, l * layer_elems, ctx->meta, n, c.n_head, cap, ctx->o_hi, o_lo, pdl, s, trace_slot(ctx, *kernels), ctx->attn_lo != 0));
+            Q(launch_gemm_ws(&t[1], &am->o_hi, &am->o_lo, ctx->x, info, d, L.b_o, n, d, d, lo, grid, sms, ctx->d_status, pdl, s, trace_slot(ctx, *kernels)));
+            Q(launch_ln_prep(ctx->x, L.ln2_g, L.ln2_b, n, d, c.ln_eps, ctx->a_hi, a_lo, ctx->h, F, info, 0, pdl, s, trace_slot(ctx, *kernels)));
+            Q(launch_gemm_ws(&t[2], &am->a_hi, &am->a_lo, ctx->h, info, F, L.b_fc, n, d, F, lo, grid, sms, ctx->d_status, pdl, s, trace_slot(ctx, *kernels)));
+            Q(launch_gelu_prep(ctx->h, n, F, ctx->h_hi, h_lo, pdl, s, trace_slot(ctx, *kernels)));
+            Q(launch_gemm_ws(&t[3], &am->h_hi, &am->h_lo, ctx->x, info, d, L.b_proj, n, F, d, lo, grid, sms, ctx->d_status, pdl, s, trace_slot(ctx, *kernels)));
         }
-        Q(launch_ln_prep(ctx->x, ctx->lnf_g, ctx->lnf_b, n, d, c.ln_eps, ctx->a_hi, a_lo, nullptr, c.vocab, info, 1, pdl, s, T()));
-        Q(launch_gemm_ws(&ctx->map_wte, &am->a_hi, &am->a_lo, nullptr, info, c.vocab, nullptr, n, d, c.vocab, lo, hgrid, sms, ctx->d_status, pdl, s, nullptr, T()));
+        Q(launch_ln_prep(ctx->x, ctx->lnf_g, ctx->lnf_b, n, d, c.ln_eps, ctx->a_hi, a_lo, nullptr, 0, info, 0, pdl, s, trace_slot(ctx, *kernels)));
+        Q(launch_gemm_ws(&ctx->map_wte, &am->a_hi, &am->a_lo, nullptr, info, c.vocab, nullptr, n, d, c.vocab, lo, hgrid, sms, ctx->d_status, pdl, s, trace_slot(ctx, *kernels)));
         ctx->trace_count = ctx->trace_kernels ? 8 * *kernels : 0;
     } else {
         for (int l = 0; l < c.n_layer; ++l) {
@@ -315,49 +279,6 @@ cudaError_t enqueue_forward(ssd_ctx *ctx, int n, int cap, const NodeList &tk, co
         Q(launch_gemm_simple(ctx->a, ctx->wte, c.dtype, nullptr, n, d, c.vocab, EPI_STORE, step.logits, s));
     }
 #undef Q
-    return cudaSuccess;
-}
-
-
-// The forward as four launches: tree preparation, embedding, the persistent all-layers kernel,
-// and the LM-head projection (which starts streaming the output embedding as SMs free up).
-cudaError_t enqueue_forward_persistent(ssd_ctx *ctx, int n, int cap, const NodeList &tk, const NodeList &pr, const StepInfo &step, int stages,
-                                       int work_bytes, size_t smem_bytes, cudaStream_t s, int *kernels) {
-    const ssd_config &c = ctx->cfg;
-    const ssd_ctx::ActMaps *am = act_maps_for(ctx, n);
-    if (!am) return cudaErrorUnknown;
-    const int d = c.d_model, F = c.d_ff, G = ctx->sm_count;
-    cudaError_t e;
-    if ((e = cudaMemsetAsync(ctx->d_ctrl, 0, 4 * sizeof(uint32_t), s)) != cudaSuccess) return e;
-    if ((e = launch_tree_prep(tk, pr, step, ctx->meta, ctx->d_info, s)) != cudaSuccess) return e;
-    if ((e = launch_embed(ctx->wte, ctx->wpe, c.dtype, ctx->meta, n, d, ctx->x, s)) != cudaSuccess) return e;
-    mega::Params p = {};
-    p.n_layer = c.n_layer; p.d = d; p.F = F; p.n_head = c.n_head; p.cap = cap; p.vocab = c.vocab;
-    p.n = n; p.n_pad = (n + 15) & ~15; p.stages = stages; p.work_bytes = work_bytes; p.use_lo = ctx->use_lo;
-    p.ln_eps = c.ln_eps;
-    p.info = ctx->d_info; p.meta = ctx->meta; p.maps = ctx->d_maps; p.vecs = ctx->d_vecs;
-    p.x = ctx->x; p.qkv_acc = ctx->qkv; p.fc_acc = ctx->h;
-    p.o_hi = ctx->o_hi; p.o_lo = ctx->o_lo; p.a_hi = ctx->a_hi; p.a_lo = ctx->a_lo;
-    p.lnf_g = ctx->lnf_g; p.lnf_b = ctx->lnf_b;
-    p.stats = ctx->d_stats; p.stats_count = ctx->d_stats_count;
-    // CTAs whose unit range reaches into output tile 0 contribute row statistics
-    auto contributors = [&](long long units, int k_tiles) {
-        uint32_t cnt = 0;
-        for (int cta = 0; cta < G; ++cta) {
-            const long long u0 = units * cta / G, u1 = units * (cta + 1) / G;
-            if (u1 > u0 && u0 < k_tiles) ++cnt;
-        }
-        return cnt;
-    };
-    p.stat_contrib_qkv = contributors((long long)((3 * d + 127) / 128) * (d / 64), d / 64);
-    p.stat_contrib_fc = contributors((long long)((F + 127) / 128) * (d / 64), d / 64);
-    p.att_part_o = ctx->d_att_part_o; p.att_part_ml = ctx->d_att_part_ml;
-    p.grid_bar = ctx->d_ctrl; p.abort_flag = ctx->d_ctrl + 1; p.grid_flag = ctx->d_ctrl + 2; p.status = ctx->d_status; p.trace = ctx->d_trace; p.trace_cta = 0;
-    if ((e = mega::launch(p, G, smem_bytes, s)) != cudaSuccess) return e;
-    if ((e = launch_gemm_ws(&ctx->map_wte, &am->a_hi, &am->a_lo, nullptr, ctx->d_info, c.vocab, nullptr, n, d, c.vocab, ctx->use_lo,
-                            head_grid_for(ctx, n), ctx->sm_count, ctx->d_status, ctx->pdl != 0, s)) != cudaSuccess)
-        return e;
-    *kernels += 4;
     return cudaSuccess;
 }
 
@@ -450,12 +371,12 @@ int ssd_create(const ssd_config *cfg, int device, void *cuda_stream, ssd_ctx **o
     memset(ctx->graphs, 0, sizeof(ctx->graphs));
     ctx->capture_stream = nullptr;
     ctx->use_graph = 1;
-    ctx->use_mega = 0;
-    ctx->use_fused = 0;
-    ctx->use_staged = 0;
-    ctx->c1_head = ctx->c2_head = ctx->d_fstats = nullptr;
-    ctx->d_tile_count = nullptr;
-    ctx->d_maps = nullptr; ctx->d_vecs = nullptr; ctx->d_stats = nullptr; ctx->d_stats_count = nullptr; ctx->d_ctrl = nullptr; ctx->d_trace = nullptr; ctx->d_att_part_o = nullptr; ctx->d_att_part_ml = nullptr;
+    ctx->use_cluster = 0;
+    ctx->attn_lo = 0;
+    ctx->cl_max = 8;
+    for (int &v : ctx->cl_size) v = 0;
+    ctx->d_stats1 = ctx->d_stats2 = nullptr;
+    ctx->d_trace = nullptr;
     ctx->sm_count = 148;
     ctx->tensor_path = cfg->dtype == SSD_DTYPE_BF16;
     ctx->use_lo = 1;
@@ -466,7 +387,7 @@ int ssd_create(const ssd_config *cfg, int device, void *cuda_stream, ssd_ctx **o
     ctx->head_grid = 0;
     ctx->a_hi = ctx->a_lo = ctx->o_hi = ctx->o_lo = ctx->h_hi = ctx->h_lo = nullptr;
     if (ctx->tensor_path) {
-        const size_t rows = (n + 15) & ~size_t(15); // operand planes hold whole 16-row boxes
+        const size_t rows = n <= 32 ? 32 : ((n + 15) & ~size_t(15)); // operand planes hold whole 16-row boxes, at least two
         A(&ctx->a_hi, rows * d); A(&ctx->a_lo, rows * d); A(&ctx->o_hi, rows * d); A(&ctx->o_lo, rows * d);
         A(&ctx->h_hi, rows * (size_t)cfg->d_ff); A(&ctx->h_lo, rows * (size_t)cfg->d_ff);
         if (rc == SSD_OK) {
@@ -479,7 +400,7 @@ int ssd_create(const ssd_config *cfg, int device, void *cuda_stream, ssd_ctx **o
             if (e == cudaSuccess) e = gemm_ws_prepare();
             if (e == cudaSuccess) e = tree_attention_mma_prepare();
             if (e == cudaSuccess) e = prep_kernels_prepare();
-            if (e == cudaSuccess) e = mega::prepare();
+            if (e == cudaSuccess) e = gemm_cl_prepare();
             if (e == cudaSuccess) e = cudaStreamCreateWithFlags(&ctx->capture_stream, cudaStreamNonBlocking);
             if (e != cudaSuccess) rc = fail_cuda(ctx, e);
             if (dev_sms > 0) ctx->sm_count = dev_sms;
@@ -561,37 +482,23 @@ int ssd_load_weights(ssd_ctx *ctx, const ssd_weights *w) {
             if (m == SSD_OK) m = make_tensor_map_bf16(&t[3], L.w_proj, d, F, 128);
         }
         if (m != SSD_OK) return m;
-        // persistent-kernel side tables: tensor maps in device memory, folded LayerNorm vectors
+        // LayerNorm-fold vectors of the cluster-reduced path, its statistics buffers, the timeline buffer
         int rc2;
-        if ((rc2 = dev_alloc(ctx, &ctx->d_maps, (size_t)4 * c.n_layer)) != SSD_OK) return rc2;
-        CU(cudaMemcpyAsync(ctx->d_maps, ctx->map_layers.data(), sizeof(CUtensorMap) * 4 * c.n_layer, cudaMemcpyHostToDevice, ctx->stream));
-        if ((rc2 = dev_alloc(ctx, &ctx->d_vecs, (size_t)c.n_layer)) != SSD_OK) return rc2;
-        if ((rc2 = dev_alloc(ctx, &ctx->d_stats, (size_t)c.n_layer * 256)) != SSD_OK) return rc2;
-        if ((rc2 = dev_alloc(ctx, &ctx->d_stats_count, (size_t)c.n_layer * 2 + 256)) != SSD_OK) return rc2;
-        if ((rc2 = dev_alloc(ctx, &ctx->d_ctrl, (size_t)4)) != SSD_OK) return rc2;
-        if ((rc2 = dev_alloc(ctx, &ctx->d_att_part_o, (size_t)8 * 64 * d)) != SSD_OK) return rc2;
-        if ((rc2 = dev_alloc(ctx, &ctx->d_att_part_ml, (size_t)8 * 64 * c.n_head * 2)) != SSD_OK) return rc2;
-        if ((rc2 = dev_alloc(ctx, &ctx->d_trace, (size_t)mega::TRACE_SLOTS)) != SSD_OK) return rc2;
-        CU(cudaMemsetAsync(ctx->d_trace, 0, sizeof(unsigned long long) * mega::TRACE_SLOTS, ctx->stream));
-        std::vector<mega::LayerVecs> hv(c.n_layer);
+        ctx->folds.assign(c.n_layer, ssd_ctx::LayerFold());
         for (int l = 0; l < c.n_layer; ++l) {
             const LayerWeights &L = ctx->layers[l];
-            float *c1q, *c2q, *c1f, *c2f;
-            if ((rc2 = dev_alloc(ctx, &c1q, 3 * d)) != SSD_OK || (rc2 = dev_alloc(ctx, &c2q, 3 * d)) != SSD_OK ||
-                (rc2 = dev_alloc(ctx, &c1f, F)) != SSD_OK || (rc2 = dev_alloc(ctx, &c2f, F)) != SSD_OK)
+            ssd_ctx::LayerFold &f = ctx->folds[l];
+            if ((rc2 = dev_alloc(ctx, &f.c1_qkv, 3 * d)) != SSD_OK || (rc2 = dev_alloc(ctx, &f.c2_qkv, 3 * d)) != SSD_OK ||
+                (rc2 = dev_alloc(ctx, &f.c1_fc, F)) != SSD_OK || (rc2 = dev_alloc(ctx, &f.c2_fc, F)) != SSD_OK)
                 return rc2;
-            CU(mega::launch_ln_fold(L.w_qkv, L.ln1_g, L.ln1_b, L.b_qkv, (int)(3 * d), (int)d, c1q, c2q, ctx->stream));
-            CU(mega::launch_ln_fold(L.w_fc, L.ln2_g, L.ln2_b, L.b_fc, (int)F, (int)d, c1f, c2f, ctx->stream));
-            hv[l] = mega::LayerVecs{L.ln1_g, c1q, c2q, L.b_o, L.ln2_g, c1f, c2f, L.b_proj};
+            CU(launch_ln_fold(L.w_qkv, L.ln1_g, L.ln1_b, L.b_qkv, (int)(3 * d), (int)d, f.c1_qkv, f.c2_qkv, ctx->stream));
+            CU(launch_ln_fold(L.w_fc, L.ln2_g, L.ln2_b, L.b_fc, (int)F, (int)d, f.c1_fc, f.c2_fc, ctx->stream));
         }
-        CU(cudaMemcpyAsync(ctx->d_vecs, hv.data(), sizeof(mega::LayerVecs) * c.n_layer, cudaMemcpyHostToDevice, ctx->stream));
-        ctx->h_vecs = hv;
-        if ((rc2 = dev_alloc(ctx, &ctx->c1_head, (size_t)c.vocab)) != SSD_OK || (rc2 = dev_alloc(ctx, &ctx->c2_head, (size_t)c.vocab)) != SSD_OK) return rc2;
-        CU(mega::launch_ln_fold(ctx->wte, ctx->lnf_g, ctx->lnf_b, nullptr, c.vocab, (int)d, ctx->c1_head, ctx->c2_head, ctx->stream));
-        if ((rc2 = dev_alloc(ctx, &ctx->d_fstats, (size_t)(2 * c.n_layer + 1) * (2 * SSD_MAX_NODES + 1))) != SSD_OK) return rc2;
-        if ((rc2 = dev_alloc(ctx, &ctx->d_tile_count, (size_t)1024)) != SSD_OK) return rc2;
-        CU(cudaMemsetAsync(ctx->d_tile_count, 0, 1024 * sizeof(int32_t), ctx->stream));
-        CU(cudaStreamSynchronize(ctx->stream)); // hv goes out of scope
+        const size_t stats_parts_max = (d + 127) / 128 > 16 ? (d + 127) / 128 : 16; // output tiles (cluster path) / CTAs per tile (self-staged path)
+        const size_t stats_floats = stats_parts_max * SSD_MAX_NODES * 2;
+        if ((rc2 = dev_alloc(ctx, &ctx->d_stats1, stats_floats)) != SSD_OK || (rc2 = dev_alloc(ctx, &ctx->d_stats2, stats_floats)) != SSD_OK) return rc2;
+        if ((rc2 = dev_alloc(ctx, &ctx->d_trace, (size_t)SSD_TRACE_SLOTS)) != SSD_OK) return rc2;
+        CU(cudaMemsetAsync(ctx->d_trace, 0, sizeof(unsigned long long) * SSD_TRACE_SLOTS, ctx->stream));
     }
     CU(cudaStreamSynchronize(ctx->stream));
     ctx->loaded = true;
@@ -669,11 +576,7 @@ int ssd_verify_tree(ssd_ctx *ctx, const int32_t *tokens, const int32_t *parent_i
     StepInfo step;
     step.n = n_nodes; step.kv_len = kv->len; step.kbase = kv->k; step.vbase = kv->v; step.logits = logits_out;
     int kernels = 0;
-    int mg_stages = 0, mg_work = 0;
-    size_t mg_smem = 0;
-    if (ctx->tensor_path && ctx->use_mega && mega::plan(n_nodes, c.d_model, c.d_ff, ctx->use_lo, ctx->sm_count, &mg_stages, &mg_work, &mg_smem)) {
-        CU(enqueue_forward_persistent(ctx, n_nodes, kv->cap, tk, pr, step, mg_stages, mg_work, mg_smem, ctx->stream, &kernels));
-    } else if (ctx->tensor_path && ctx->use_graph) {
+    if (ctx->tensor_path && ctx->use_graph) {
         ssd_ctx::ForwardGraph &fg = ctx->graphs[n_nodes];
         if (!fg.exec) {
             rc = capture_forward(ctx, n_nodes, kv->cap, tk, pr, step);
@@ -804,9 +707,12 @@ int ssd_set_tuning(ssd_ctx *ctx, int32_t knob, int32_t value) {
     case SSD_TUNE_GEMM_CTAS: if (value < 0 || value > 4096) return SSD_ERR_BAD_ARG; ctx->gemm_grid = value; break;
     case SSD_TUNE_KERNEL_TRACE: if (value != 0 && value != 1) return SSD_ERR_BAD_ARG; ctx->trace_kernels = value; ctx->trace_count = 0; break;
     case SSD_TUNE_HEAD_CTAS: if (value < 0 || value > 4096) return SSD_ERR_BAD_ARG; ctx->head_grid = value; break;
-    case SSD_TUNE_FUSED_TAILS: if (value != 0 && value != 1) return SSD_ERR_BAD_ARG; ctx->use_fused = value; break;
-    case SSD_TUNE_SELF_STAGED: if (value != 0 && value != 1) return SSD_ERR_BAD_ARG; ctx->use_staged = value; break;
-    case SSD_TUNE_PERSISTENT: if (value != 0 && value != 1) return SSD_ERR_BAD_ARG; ctx->use_mega = value; break;
+    case SSD_TUNE_CLUSTER_REDUCE: if (value != 0 && value != 1) return SSD_ERR_BAD_ARG; ctx->use_cluster = value; break;
+    case SSD_TUNE_ATTN_LOW_PLANE: if (value != 0 && value != 1) return SSD_ERR_BAD_ARG; ctx->attn_lo = value; break;
+    case SSD_TUNE_CLUSTER_MAX: if (value < 1 || value > 16) return SSD_ERR_BAD_ARG; ctx->cl_max = value; break;
+    case SSD_TUNE_CLUSTER_QKV: case SSD_TUNE_CLUSTER_O: case SSD_TUNE_CLUSTER_FC: case SSD_TUNE_CLUSTER_PROJ:
+        if (value < 0 || value > 16) return SSD_ERR_BAD_ARG;
+        ctx->cl_size[knob - SSD_TUNE_CLUSTER_QKV] = value; break;
     default: return SSD_ERR_BAD_ARG;
     }
     DeviceGuard g(ctx->device);
@@ -822,15 +728,11 @@ int ssd_get_phase_trace(ssd_ctx *ctx, uint64_t *out_ns, int32_t capacity, int32_
     if (!ctx->d_trace) return SSD_OK;
     DeviceGuard g(ctx->device);
     if (!g.ok) return SSD_ERR_CUDA;
-    std::vector<unsigned long long> h(mega::TRACE_SLOTS);
-    CU(cudaMemcpyAsync(h.data(), ctx->d_trace, sizeof(unsigned long long) * mega::TRACE_SLOTS, cudaMemcpyDeviceToHost, ctx->stream));
+    std::vector<unsigned long long> h(SSD_TRACE_SLOTS);
+    CU(cudaMemcpyAsync(h.data(), ctx->d_trace, sizeof(unsigned long long) * SSD_TRACE_SLOTS, cudaMemcpyDeviceToHost, ctx->stream));
     CU(cudaStreamSynchronize(ctx->stream));
     int n = 0;
-    if (ctx->trace_count > 0) { // per-launch timeline: eight slots per kernel, unused ones zero
-        for (; n < ctx->trace_count && n < mega::TRACE_SLOTS && n < capacity; ++n) out_ns[n] = h[n];
-    } else {
-        while (n < mega::TRACE_SLOTS && n < capacity && h[n] != 0ull) { out_ns[n] = h[n]; ++n; }
-    }
+    for (; n < ctx->trace_count && n < SSD_TRACE_SLOTS && n < capacity; ++n) out_ns[n] = h[n]; // eight slots per kernel, unused ones zero
     *count = n;
     return SSD_OK;
 }

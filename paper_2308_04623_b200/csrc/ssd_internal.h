@@ -8,6 +8,7 @@
 
 #define SSD_MAX_NODES 256
 #define SSD_ANC_WORDS 4 /* 256 nodes / 64 bits */
+#define SSD_TRACE_SLOTS 4096 /* timeline buffer: eight 64-bit stamps per launch */
 
 // Small host arrays travel to the device as kernel arguments: no staging buffer, no copy to
 // wait for, and the call may return before the kernel runs.
@@ -48,10 +49,7 @@ cudaError_t launch_tree_prep(const NodeList &tokens, const NodeList &parent, con
 // fills the argument array of that node.
 const void *tree_prep_kernel_address();
 cudaError_t launch_embed(const void *wte, const void *wpe, int dtype, const TreeMeta &m, int n, int d, float *x, cudaStream_t s);
-cudaError_t launch_embed_fold(const void *wte, const void *wpe, const TreeMeta &m, int n, int d, const float *gain, float *x, void *plane_hi,
-                              void *plane_lo, float *stats, int stats_floats, float *qkv, int qkv_cols, float *fc, int fc_cols,
-                              cudaStream_t s);
-cudaError_t launch_zero_logits(const StepInfo *info, int n, int vocab, bool pdl, cudaStream_t s);
+cudaError_t launch_zero_logits(const StepInfo *info, int n, int vocab, cudaStream_t s);
 cudaError_t launch_layernorm(const float *x, const float *g, const float *b, int n, int d, float eps, float *out, cudaStream_t s);
 // y[n, out] (+)= epilogue(a[n, K] . W[out, K]^T + bias)
 cudaError_t launch_gemm_simple(const float *a, const void *W, int dtype, const float *bias, int n, int K, int out, int epilogue,
@@ -74,44 +72,6 @@ cudaError_t launch_gelu_prep(const float *acc, int n, int F, __nv_bfloat16 *h_hi
 // Tensor maps are opaque 128-byte objects (CUtensorMap) built on the host.
 struct alignas(64) TensorMap { unsigned char bytes[128]; };
 int make_tensor_map_bf16(void *map_out, const void *base, uint64_t rows, uint64_t cols, uint32_t box_rows);
-// Optional work fused into the projection kernel.
-//  * fold: the projection ran on x * gain; its epilogue applies rstd * (acc - mean * c1) + c2 with the row
-//    statistics `stats_in` ([n][2]: sum, sum of squares of x) - the LayerNorm in front of the projection.
-//  * tail, done by whichever CTA adds the LAST partial sum to an output tile (no extra launch):
-//      TAIL_LN_PLANES   y is the residual stream x: write bf16 hi/lo planes of x * gain (the operand of the next
-//                       LayerNorm-folded projection), add the rows' sum / sum of squares over the tile's columns
-//                       to stats_out, and clear a share of the `zero` buffer;
-//      TAIL_GELU_PLANES y holds raw FC accumulators: write planes of gelu(rstd * (acc - mean * c1) + c2) and clear
-//                       the accumulators for the next layer.
-enum { TAIL_NONE = 0, TAIL_LN_PLANES = 1, TAIL_GELU_PLANES = 2 };
-//  * src_mode: where operand B (the activations) comes from.  SRC_TMA: bf16 planes through the tensor maps.
-//    SRC_LN_GAIN / SRC_GELU: the CTA converts `src` ([n, src_ld] fp32) itself, as src * gain (the LayerNorm is then
-//    applied by whoever consumes the accumulators: `fold` here, or the attention kernel) or gelu(src).  With
-//    SRC_LN_GAIN and stats_out set, the rows' sum / sum of squares go to stats_out and the contributing CTAs count
-//    themselves on stats_counter; a kernel with `fold` and stats_counter set waits for that count.  Needs one
-//    pipeline stage per unit of a CTA (gemm_ws_can_self_stage).
-//  * clear: an fp32 buffer of clear_floats (a multiple of 4) values that the kernel zeroes after the kernels before it
-//    have completed.
-enum { SRC_TMA = 0, SRC_LN_GAIN = 1, SRC_GELU = 2 };
-struct GemmFusion {
-    int fold, tail;
-    const float *stats_in, *c1, *c2; // fold / TAIL_GELU_PLANES
-    float inv_d, eps;
-    const float *gain;               // TAIL_LN_PLANES
-    float *stats_out;                // TAIL_LN_PLANES: [n][2]
-    __nv_bfloat16 *plane_hi, *plane_lo;
-    int plane_ld;
-    float *zero;                     // TAIL_LN_PLANES: [n, zero_cols] accumulators to clear (may be null)
-    int zero_cols;
-    int32_t *tile_count;             // [n_tiles] arrival counters, zero at rest
-    int src_mode;                    // SRC_*
-    const float *src;
-    int src_ld;
-    int *stats_counter;
-    float *clear;
-    size_t clear_floats;
-};
-bool gemm_ws_can_self_stage(int n, int K, int out, int use_lo, int grid, int sm_count);
 cudaError_t gemm_ws_prepare();
 cudaError_t prep_kernels_prepare();
 // y[n, ldy] += X[n, K] . W[out, K]^T (+ bias once).  map_w: weights [out, K], boxes of 128 rows; map_hi / map_lo:
@@ -120,7 +80,40 @@ cudaError_t prep_kernels_prepare();
 // half an SM's shared memory.
 cudaError_t launch_gemm_ws(const void *map_w, const void *map_hi, const void *map_lo, float *y, const StepInfo *info, int ldy,
                            const float *bias, int n, int K, int out, int use_lo, int grid, int sm_count, int32_t *status, bool pdl,
-                           cudaStream_t s, const GemmFusion *fusion = nullptr, unsigned long long *trace = nullptr);
+                           cudaStream_t s, unsigned long long *trace = nullptr);
+// ---- projection with the split-K sums reduced inside a thread-block cluster (trees of up to 64 nodes) ----
+// What the epilogue does with the finished sums acc[i, o] (see k_gemm_cl.cu):
+enum { MODE_FOLD_STORE = 0, MODE_FOLD_GELU = 1, MODE_RESIDUAL = 2 };
+struct GemmClEpilogue {
+    int mode;
+    // MODE_FOLD_*: statistics of the LayerNorm in front of the projection as `stats_parts` partial
+    // (sum, sum of squares) pairs per row, [part][SSD_MAX_NODES][2]; c1 = W gain, c2 = W beta + bias
+    const float *stats_in;
+    int stats_parts;
+    const float *c1, *c2;
+    float inv_d, eps;
+    float *y;               // MODE_FOLD_STORE: output [n, ldy]; MODE_RESIDUAL: the residual stream, updated in place
+    int ldy;
+    const float *bias;      // MODE_RESIDUAL
+    const float *gain;      // MODE_RESIDUAL: gain of the next LayerNorm, planes = x * gain (null: no planes)
+    __nv_bfloat16 *plane_hi, *plane_lo; // MODE_FOLD_GELU / MODE_RESIDUAL: bf16 operand planes [rows, plane_ld] of the next projection
+    int plane_ld;
+    float *stats_out;       // MODE_RESIDUAL: [output tile][SSD_MAX_NODES][2]
+};
+cudaError_t gemm_cl_prepare();
+bool gemm_cl_supports(int n, int d_model);
+int gemm_cl_n_pad(int n);
+int gemm_cl_cluster_size(int n, int K, int out, int slots, int max_cluster);
+cudaError_t launch_gemm_cl(const void *map_w, const void *map_hi, const void *map_lo, int n, int K, int out, int use_lo, int cluster,
+                           bool two_per_sm, const GemmClEpilogue &ep, int32_t *status, bool pdl, cudaStream_t s,
+                           unsigned long long *trace = nullptr);
+// x = wte[token] + wpe[pos] with the bf16 hi/lo planes of x * gain and the rows' (sum, sum of squares) as statistics part 0
+cudaError_t launch_embed_planes(const void *wte, const void *wpe, const TreeMeta &m, int n, int d, const float *gain, float *x, void *plane_hi,
+                                void *plane_lo, float *stats, cudaStream_t s);
+// c1[o] = sum_k g[k] W[o, k], c2[o] = sum_k beta[k] W[o, k] + bias[o] (bias may be null): the vectors that fold a LayerNorm into
+// the projection behind it
+cudaError_t launch_ln_fold(const void *W, const float *g, const float *beta, const float *bias, int out, int K, float *c1, float *c2, cudaStream_t s);
+
 // Moves slot kv_len + path[j] -> kv_len + j for every layer, K and V, head.
 // (bf16 caches keep V transposed, [H, 64, cap]; fp32 caches keep V like K, [H, cap, 64].)
 cudaError_t launch_kv_commit(void *kbase, void *vbase, int dtype, int n_layer, int n_head, int cap, int kv_len, const NodeList &path,
@@ -132,8 +125,7 @@ size_t tree_attention_mma_smem(int n);
 cudaError_t tree_attention_mma_prepare();
 cudaError_t launch_tree_attention_mma(const float *qkv, const StepInfo *info, size_t layer_offset_elems, const TreeMeta &m, int n, int n_head,
                                       int cap, __nv_bfloat16 *o_hi, __nv_bfloat16 *o_lo, bool pdl, cudaStream_t s,
-                                      const float *fold_stats = nullptr, const float *fold_c1 = nullptr, const float *fold_c2 = nullptr,
-                                      float fold_eps = 0.f, unsigned long long *trace = nullptr);
+                                      unsigned long long *trace = nullptr, bool lo_pairs = true);
 
 #define SSD_ACC_SUPPORT 1024
 struct AcceptScratch {

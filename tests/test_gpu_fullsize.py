@@ -15,15 +15,13 @@ pytestmark = pytest.mark.gpu
 TOL_BF16 = 3e-2
 
 
-def _run(name, P, trees, seed=0, chunk=256, persistent=False):
+def _run(name, P, trees, seed=0, chunk=256):
     from tests import gpu_util
     import paper_2308_04623_b200 as ssd
     p = gpu_util.Pair(name, seed=seed)
     worst = {}
     fragile = 0
     try:
-        if persistent:
-            p.ctx.set_tuning(ssd.SSD_TUNE_PERSISTENT, 1)
         rng = np.random.default_rng(1002)
         p.prefill(ssd_synth.uniform_tokens(P, p.V, rng), chunk=chunk)
         for label, tokens, parent in trees(p, rng):
@@ -62,13 +60,6 @@ def test_gpt2_large_shape_256_prefix_trees_16_32_64():
         for n, br in ((32, (4, 2, 2, 1, 1)), (16, (4, 2, 2, 1, 1)), (64, (4, 2, 2, 2, 1, 1))):
             yield "n=%d" % n, ssd_synth.uniform_tokens(n, p.V, rng), ssd_synth.tree_branching(n, br)
     _run("gpt2_large", 256, trees)
-
-
-def test_gpt2_large_shape_persistent_kernel():
-    def trees(p, rng):
-        for n, br in ((32, (4, 2, 2, 1, 1)), (64, (4, 2, 2, 2, 1, 1))):
-            yield "n=%d" % n, ssd_synth.uniform_tokens(n, p.V, rng), ssd_synth.tree_branching(n, br)
-    _run("gpt2_large", 256, trees, persistent=True)
 
 
 def test_gpt2_small_shape_stage_two_trigram_tree():

@@ -482,38 +482,18 @@ def test_bf16_steps_with_commit(util):
         p.close()
 
 
-# --------------------------------------------------------------------------- fused tails (opt-in)
-@pytest.mark.parametrize("name,n", [("tiny_bf16", 7), ("tiny_bf16", 40), ("ragged_bf16", 33), ("tiny_bf16", 150)])
-def test_fused_tails_path_logits_and_steps(name, n, util, ssd):
-    """Five launches per layer: LayerNorms folded into the projections, operand planes written by the CTA that
-    completes an output tile.  Same results within the bf16 tolerance, over two committed steps."""
+# --------------------------------------------------------------------------- cluster-reduced projections, CTA counts
+@pytest.mark.parametrize("name,n,cmax", [("tiny_bf16", 1, 8), ("tiny_bf16", 7, 1), ("tiny_bf16", 16, 2), ("tiny_bf16", 40, 8), ("ragged_bf16", 33, 3),
+                                         ("tiny_bf16", 64, 4), ("ragged_bf16", 48, 5), ("tiny_bf16", 31, 16), ("ragged_bf16", 17, 7)])
+def test_cluster_reduced_path_cluster_sizes_and_steps(name, n, cmax, util, ssd):
+    """Five launches per layer: split-K partial sums reduced inside a thread-block cluster, LayerNorms folded, GELU and
+    the residual additions in the epilogues.  Every cluster size (1 = no split, odd sizes with uneven column chunks, the
+    non-portable 16) gives logits within the bf16 tolerance, bit-identical from run to run, over two committed steps; the
+    launch count shows that the path ran; the 8-launch path gives the same logits within twice the tolerance's noise."""
     p = util.Pair(name, seed=9, qk_gain=3.0)
     try:
-        p.ctx.set_tuning(ssd.SSD_TUNE_FUSED_TAILS, 1)
-        rng = np.random.default_rng(200 + n)
-        p.prefill(ssd_synth.uniform_tokens(37, p.V, rng), chunk=32)
-        for step in range(2):
-            parent = ssd_synth.tree_random(n, 6, rng)
-            tokens = ssd_synth.uniform_tokens(n, p.V, rng)
-            got, want, buf = p.verify(tokens, parent)
-            assert np.isfinite(got).all()
-            assert np.abs(got - want).max() <= TOL_BF16
-            path, nxt = p.ctx.accept_tree(buf.data_ptr(), None, tokens, parent)
-            p.commit(path)
-        assert p.ctx.device_status() == 0
-    finally:
-        p.close()
-
-
-# --------------------------------------------------------------------------- self-staged operands (opt-in), CTA counts
-@pytest.mark.parametrize("name,n", [("tiny_bf16", 1), ("tiny_bf16", 7), ("tiny_bf16", 40), ("ragged_bf16", 33), ("tiny_bf16", 150)])
-def test_self_staged_path_logits_and_steps(name, n, util, ssd):
-    """Five launches per layer: the projections behind a LayerNorm or the GELU convert their activations themselves,
-    the LayerNorm being applied by the consumer of the accumulators.  Same results within the bf16 tolerance, over
-    two committed steps; the launch count shows that the path ran."""
-    p = util.Pair(name, seed=9, qk_gain=3.0)
-    try:
-        p.ctx.set_tuning(ssd.SSD_TUNE_SELF_STAGED, 1)
+        p.ctx.set_tuning(ssd.SSD_TUNE_CLUSTER_REDUCE, 1)
+        p.ctx.set_tuning(ssd.SSD_TUNE_CLUSTER_MAX, cmax)
         rng = np.random.default_rng(300 + n)
         p.prefill(ssd_synth.uniform_tokens(37, p.V, rng), chunk=32)
         for step in range(2):
@@ -521,11 +501,26 @@ def test_self_staged_path_logits_and_steps(name, n, util, ssd):
             tokens = ssd_synth.uniform_tokens(n, p.V, rng)
             before = p.ctx.kernel_launches()
             got, want, buf = p.verify(tokens, parent)
-            assert p.ctx.kernel_launches() - before == 2 + 5 * p.cfg["n_layer"] + 2
+            assert p.ctx.kernel_launches() - before == 3 + 5 * p.cfg["n_layer"] + 2
             assert np.isfinite(got).all()
             assert np.abs(got - want).max() <= TOL_BF16
+            if step == 0:
+                again, _, _ = p.verify(tokens, parent)
+                # the layers are reproducible bit for bit; the LM head still adds its stream-K partial sums at L2
+                assert np.abs(again - got).max() <= 1e-5, np.abs(again - got).max()
+                p.ctx.set_tuning(ssd.SSD_TUNE_CLUSTER_REDUCE, 0)
+                before = p.ctx.kernel_launches()
+                plain, _, _ = p.verify(tokens, parent)
+                assert p.ctx.kernel_launches() - before == 3 + 8 * p.cfg["n_layer"] + 2
+                assert np.abs(plain - want).max() <= TOL_BF16
+                p.ctx.set_tuning(ssd.SSD_TUNE_CLUSTER_REDUCE, 1)
+                got, want, buf = p.verify(tokens, parent)
             path, nxt = p.ctx.accept_tree(buf.data_ptr(), None, tokens, parent)
             p.commit(path)
+            for l in range(p.cfg["n_layer"]):
+                for which_kv in (0, 1):
+                    a = p.ctx.kv_read(p.kv, l, which_kv, 0, len(p.kv))
+                    assert np.abs(a - p.okv.read(l, which_kv, 0, len(p.kv))).max() <= 3e-2
         assert p.ctx.device_status() == 0
     finally:
         p.close()
@@ -534,9 +529,11 @@ def test_self_staged_path_logits_and_steps(name, n, util, ssd):
 @pytest.mark.parametrize("ctas", [1, 37, 148, 296, 500])
 def test_projection_cta_counts_give_the_same_logits(ctas, util, ssd):
     """The (output tile, k tile) units of a projection are cut into one contiguous range per CTA, whatever the CTA
-    count (one CTA, fewer CTAs than SMs, one or two per SM, more CTAs than units for the small matrices)."""
+    count (one CTA, fewer CTAs than SMs, one or two per SM, more CTAs than units for the small matrices); on the
+    cluster-reduced path the count bounds the clusters' sizes instead."""
     p = util.Pair("ragged_bf16", seed=4, qk_gain=3.0)
     try:
+        p.ctx.set_tuning(ssd.SSD_TUNE_CLUSTER_REDUCE, ctas % 2)
         p.ctx.set_tuning(ssd.SSD_TUNE_GEMM_CTAS, ctas)
         p.ctx.set_tuning(ssd.SSD_TUNE_HEAD_CTAS, max(1, ctas // 2))
         rng = np.random.default_rng(77)
@@ -564,45 +561,15 @@ def test_kernel_timeline_has_eight_ordered_stamps_per_launch(util, ssd):
         before = p.ctx.kernel_launches()
         got, _, _ = p.verify(tokens, parent)
         kernels = p.ctx.kernel_launches() - before
-        assert np.abs(got - base).max() <= 1e-4   # (the order of the fp32 reductions at L2 differs from run to run)
+        # (the order of the fp32 reductions at L2 differs from run to run, and a last-bit difference can move a query or a
+        #  softmax weight across a bf16 rounding boundary inside the attention kernel)
+        assert np.abs(got - base).max() <= 1e-3
         t = p.ctx.phase_trace().astype(np.int64)
         assert len(t) == 8 * kernels
-        t = t.reshape(kernels, 8)[2:]          # (the two set-up kernels are not traced)
+        t = t.reshape(kernels, 8)[3:]          # (the three set-up kernels are not traced)
         assert (t[:, 0] > 0).all() and (t[:, 0] <= t[:, 1]).all() and (t[:, 1] <= t[:, 2]).all() and (t[:, 2] <= t[:, 6]).all()
         assert (np.diff(t[:, 1]) >= 0).all()   # dependencies are met in launch order
         p.ctx.set_tuning(ssd.SSD_TUNE_KERNEL_TRACE, 0)
-        assert p.ctx.device_status() == 0
-    finally:
-        p.close()
-
-
-# --------------------------------------------------------------------------- persistent all-layers kernel (opt-in)
-@pytest.mark.parametrize("name,n", [("tiny_bf16", 1), ("tiny_bf16", 15), ("tiny_bf16", 32), ("tiny_bf16", 33), ("tiny_bf16", 64),
-                                    ("ragged_bf16", 24), ("ragged_bf16", 48)])
-def test_persistent_kernel_logits_and_steps(name, n, util, ssd):
-    """The same forward as one cooperative launch (trees of up to 64 nodes): logits within the bf16 tolerance,
-    scratch K/V written, and a committed step followed by a second verify."""
-    p = util.Pair(name, seed=7, qk_gain=3.0)
-    try:
-        p.ctx.set_tuning(ssd.SSD_TUNE_PERSISTENT, 1)
-        rng = np.random.default_rng(100 + n)
-        p.prefill(ssd_synth.uniform_tokens(45, p.V, rng), chunk=16)
-        for step in range(2):
-            parent = ssd_synth.tree_random(n, 6, rng)
-            tokens = ssd_synth.uniform_tokens(n, p.V, rng)
-            launches = p.ctx.kernel_launches()
-            got, want, buf = p.verify(tokens, parent)
-            assert p.ctx.kernel_launches() - launches == 4  # tree prep, embed, persistent forward, LM head
-            assert np.isfinite(got).all()
-            assert np.abs(got - want).max() <= TOL_BF16
-            path, nxt = p.ctx.accept_tree(buf.data_ptr(), None, tokens, parent)
-            opath, onxt, _ = ssd_oracle.accept_tree(got.astype(np.float32), None, tokens, parent, mode=0)
-            assert (path, nxt) == (opath, onxt)
-            p.commit(path)
-            for l in range(p.cfg["n_layer"]):
-                for which_kv in (0, 1):
-                    a = p.ctx.kv_read(p.kv, l, which_kv, 0, len(p.kv))
-                    assert np.abs(a - p.okv.read(l, which_kv, 0, len(p.kv))).max() <= 3e-2
         assert p.ctx.device_status() == 0
     finally:
         p.close()

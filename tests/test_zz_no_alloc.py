@@ -67,7 +67,11 @@ def test_noalloc_entry_point_matches_regular_entry_point_twice_in_a_row(V):
             lg = torch.from_numpy(logits).cuda()
             dp = torch.from_numpy(draft).cuda()
             # one warm call (symbol look-up, lazy module load), then the free device memory must not move
+            # (the regular entry point is warmed too: it grows its own per-context scratch on its first sampling call)
             _call_noalloc(ssd, lg, dp, tokens, parent, V, ssd.SSD_SAMPLING, 1, 0, 1.0, 0)
+            _call_noalloc(ssd, lg, dp, tokens, parent, V, ssd.SSD_GREEDY, 1, 0, 1.0, 0)
+            _call_regular(ssd, ctx, lg, dp, tokens, parent, ssd.SSD_SAMPLING, 1, 0, 1.0, 50)
+            _call_regular(ssd, ctx, lg, dp, tokens, parent, ssd.SSD_GREEDY, 1, 0, 1.0, 0)
             torch.cuda.synchronize()
             free_before = torch.cuda.mem_get_info()[0]
             for mode, T, k in ((ssd.SSD_GREEDY, 1.0, 0), (ssd.SSD_SAMPLING, 1.0, 0), (ssd.SSD_SAMPLING, 0.75, 50)):
