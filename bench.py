@@ -1,26 +1,36 @@
 #!/usr/bin/env python
 """Benchmark of the tree-verification hot path (verify -> accept -> commit) on B200.
 
-    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl reference]
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl reference] [--no-sweep]
 
 One step = one pass of the whole hot path over one synthetic batch: ssd_verify_tree of a
 32-node tree against a 256-token cache on the GPT-2-Large shape (36 x 1280, vocab 50257, bf16,
 random N(0, 0.02) weights), ssd_accept_tree on the produced logits, ssd_kv_commit of the accepted
 path; the cache is then rolled back (host-side length only) so that every step sees the same
-prefix length.  Token ids are re-drawn for every step.  Prints ONE JSON line.
+prefix length.  A few token sets are prepared before the timed region: random ids, with the
+verifier's own arg-max token planted on each child with probability 0.6 (level by level, from
+untimed verifications of the same prefix), so that the timed steps accept paths of several nodes
+and the commit really gathers rows.  Prints ONE JSON line.
+
+At one GPU the line also carries a `sweep` measured in the same process: the 16- and 64-node
+trees on the same model, the stage-two verification of the GPT-2-small-shaped draft (512-token
+prefix, eight-node trigram tree) with a warm L2 and with an L2-evicting pass between steps, and the
+GPT-2-XL-shaped model over tree sizes 8..256 with the fractions of the HBM and tensor-core
+roofs and the tree size at which the tensor bound overtakes the HBM bound.
 
 N > 1 runs N independent replicas (one process per GPU, no data-path collective): the path is a
-single sequence at batch 1 and does not shard.
+single sequence at batch 1 and does not shard.  Without torchrun's environment the script starts
+the N replica processes itself.
 """
 from __future__ import annotations
 
 import argparse
 import json
 import os
+import socket
 import subprocess
 import sys
 import tempfile
-import threading
 import time
 
 import numpy as np
@@ -34,9 +44,10 @@ import ssd_synth  # noqa: E402
 METRIC = "GPT-2-L-shape tree-verify us/step (verify+accept+commit)"
 UNIT = "us/step"
 NOMINAL_HBM_GBS = 8000.0
-# DRAM bytes (read + write) of one forward of the metric's workload, from the ncu launch list in
-# profiles/bench_step_gpt2_large_n32_launch_list.md (per step, like `achieved`)
-NCU_TRAFFIC_BYTES = {("gpt2_large", 32, 256): 1758.3e6}
+PLANT_PROBABILITY = 0.6
+# DRAM bytes (read + write) of one forward of the metric's workload: sum over the ncu launch list in
+# profiles/bench_step_gpt2_large_n32_launch_list.md (per forward, like `achieved`)
+NCU_TRAFFIC_BYTES = {("gpt2_large", 32, 256): 1743.4e6}
 
 
 def measured_peaks():
@@ -110,21 +121,15 @@ def workload(args):
     return cfg, parent
 
 
-def oracle_sample_step(cfg, weights, parent, sample_nodes, sample_prefix, rng):
-    """One oracle step on a bounded sample of the workload; returns a closure that runs it."""
-    from oracle import ssd_oracle
-    model = ssd_oracle.Model(cfg, weights)
-    kv = model.new_kv()
-    kv.prefill(ssd_synth.uniform_tokens(sample_prefix, cfg["vocab"], rng), chunk=sample_prefix)
-    par = parent[:sample_nodes].copy()
+def gemm_flops(cfg: dict, n_nodes: int) -> float:
+    """Multiply-add flops of the dense projections of one forward over n_nodes rows."""
+    d, F, L, V = cfg["d_model"], cfg["d_ff"], cfg["n_layer"], cfg["vocab"]
+    return 2.0 * n_nodes * (L * (4 * d * d + 2 * d * F) + V * d)
 
-    def step():
-        tokens = ssd_synth.uniform_tokens(sample_nodes, cfg["vocab"], rng)
-        logits = kv.verify_tree(tokens, par)
-        path, nxt, _ = ssd_oracle.accept_tree(logits, None, tokens, par, mode=0)
-        kv.commit(path)
-        kv.rollback(sample_prefix)
-    return step
+
+def percentiles(values) -> dict:
+    v = np.asarray(values, dtype=np.float64)
+    return {"median": float(np.median(v)), "p10": float(np.percentile(v, 10)), "p90": float(np.percentile(v, 90)), "mean": float(v.mean())}
 
 
 def max_over_ranks(values, device="cuda"):
@@ -143,48 +148,275 @@ def replica_value(ms_per_step: float, world: int) -> float:
     return ms_per_step * 1e3 / world
 
 
+def replica_env(rank: int, world: int, port: int) -> dict:
+    """Environment of one replica process started by this script (what torchrun would have set)."""
+    env = dict(os.environ)
+    env.update(RANK=str(rank), LOCAL_RANK=str(rank), WORLD_SIZE=str(world), MASTER_ADDR="127.0.0.1", MASTER_PORT=str(port))
+    return env
+
+
+def spawn_replicas(world: int, argv, script=None) -> int:
+    """Start `world` copies of this script, one per GPU; rank 0's output (the JSON line) is this process's output."""
+    with socket.socket() as s:
+        s.bind(("127.0.0.1", 0))
+        port = s.getsockname()[1]
+    procs = [subprocess.Popen([sys.executable, script or os.path.abspath(__file__)] + list(argv), env=replica_env(r, world, port),
+                              stdout=None if r == 0 else subprocess.DEVNULL) for r in range(world)]
+    rc = 0
+    for p in procs:
+        rc = p.wait() or rc
+    return rc
+
+
 def omp_threads() -> int:
     v = os.environ.get("OMP_NUM_THREADS")
     return int(v) if v and v.isdigit() else (os.cpu_count() or 1)
 
 
+# ------------------------------------------------------------------------------------------------
+# CPU oracle (the reference arm and the cpu_baseline leg): the only code here that touches oracle/
+# ------------------------------------------------------------------------------------------------
+def oracle_steps(cfg, weights, parent, prefix_len, rng, max_steps, warmup, budget_s):
+    """Times full oracle steps (verify + accept + commit of the whole tree at the full prefix).  Returns the step times (s)."""
+    from oracle import ssd_oracle
+    model = ssd_oracle.Model(cfg, weights)
+    kv = model.new_kv()
+    V, n = cfg["vocab"], len(parent)
+    deadline = time.time() + budget_s
+    kv.prefill(ssd_synth.uniform_tokens(prefix_len, V, rng), chunk=min(prefix_len, 256) or 1)
+
+    def step():
+        tokens = ssd_synth.uniform_tokens(n, V, rng)
+        logits = kv.verify_tree(tokens, parent)
+        path, nxt, _ = ssd_oracle.accept_tree(logits, None, tokens, parent, mode=0)
+        kv.commit(path)
+        kv.rollback(prefix_len)
+
+    for _ in range(warmup):
+        if time.time() > deadline:
+            break
+        step()
+    times = []
+    for _ in range(max_steps):
+        t0 = time.perf_counter()
+        step()
+        times.append(time.perf_counter() - t0)
+        if time.time() > deadline:
+            break
+    return times
+
+
 def run_reference(args):
-    """The CPU oracle, as it stands, timed on the host cores (rank 0 only)."""
+    """The CPU oracle, as it stands, timed on the host cores (rank 0 only) on the metric's full workload."""
     if int(os.environ.get("RANK", "0")) != 0:
         return
     cfg, parent = workload(args)
     rng = np.random.default_rng(1002)
     weights = ssd_synth.make_weights(cfg, seed=0)
-    sn, sp = min(args.ref_nodes, args.nodes), args.ref_prefix
-    step = oracle_sample_step(cfg, weights, parent, sn, sp, rng)
-    scale = args.nodes / sn
-    budget = time.time() + args.ref_budget_s
-    for _ in range(args.warmup):
-        step()
-        if time.time() > budget:
-            break
-    times = []
-    for _ in range(args.steps):
-        t0 = time.perf_counter()
-        step()
-        times.append(time.perf_counter() - t0)
-        if time.time() > budget and len(times) >= 1:
-            break
-    us = float(np.mean(times)) * 1e6 * scale
-    sample = ("oracle verify+accept+commit on the first %d nodes of the %d-node tree, prefix %d instead of %d; time scaled by %g "
-              "(projection cost is linear in nodes); %d of %d steps timed" % (sn, args.nodes, sp, args.prefix, scale, len(times), args.steps))
+    times = oracle_steps(cfg, weights, parent, args.prefix, rng, args.steps, min(args.warmup, 1), args.ref_budget_s)
+    us = float(np.median(times)) * 1e6
+    sample = ("full oracle steps (verify + accept + commit of the %d-node tree at prefix %d), median of %d of %d steps "
+              "(time budget %g s)" % (args.nodes, args.prefix, len(times), args.steps, args.ref_budget_s))
     line = {"impl": "reference", "metric": METRIC, "value": us, "unit": UNIT, "n_gpus": args.gpus, "steps": args.steps,
             "warmup": args.warmup, "ms_per_step": us / 1e3, "higher_is_better": False, "scaling": "weak", "vs_baseline": None,
             "dtype": "f64", "data": "synthetic",
-            "config": {"workload": "%s verify n=%d prefix=%d (CPU oracle on a bounded sample)" % (args.model, args.nodes, args.prefix)},
+            "config": {"workload": "%s verify n=%d prefix=%d, greedy accept, commit (CPU oracle)" % (args.model, args.nodes, args.prefix)},
             "cpu_baseline": {"value": us, "unit": UNIT, "cores": omp_threads(), "kind": "oracle", "sample": sample},
             "e2e": {"value": us, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0}}
     print(json.dumps(line), flush=True)
 
 
+# ------------------------------------------------------------------------------------------------
+# GPU arm
+# ------------------------------------------------------------------------------------------------
+class Runner:
+    """One model on the device with a prefilled cache; times steps of a given tree."""
+
+    def __init__(self, model, prefix_len, device, tune=(), seed=0, rng_seed=1002):
+        import torch
+        import paper_2308_04623_b200 as ssd
+        self.torch, self.ssd = torch, ssd
+        self.cfg = ssd_synth.config(model)
+        self.model, self.P, self.V = model, prefix_len, self.cfg["vocab"]
+        self.rng = np.random.default_rng(rng_seed)
+        self.weights = ssd_synth.make_weights(self.cfg, seed=seed)
+        self.stream = torch.cuda.current_stream()
+        self.ctx = ssd.Context(self.cfg, device=device, stream=self.stream.cuda_stream)
+        self.ctx.load_weights(ssd_synth.bf16_bits(self.weights) if self.cfg["dtype"] == "bf16" else self.weights)
+        for spec in tune:
+            knob, value = spec.split("=")
+            self.ctx.set_tuning(int(knob), int(value))
+        self.kv = self.ctx.new_kv()
+        self.logits = torch.empty((256, self.V), dtype=torch.float32, device="cuda")
+        self.prefix = ssd_synth.uniform_tokens(prefix_len, self.V, self.rng)
+        for s in range(0, prefix_len, 256):  # prefix through hot-path calls only: chain trees, every node committed
+            t = self.prefix[s:s + 256]
+            self.ctx.verify_tree(t, ssd_synth.tree_chain(len(t)), self.kv, self.logits.data_ptr())
+            self.ctx.kv_commit(self.kv, np.arange(len(t), dtype=np.int32))
+        self.srng = ssd.binding.ssd_rng(1, 0)
+        self.evict = None
+
+    def planted_tokens(self, parent, sets, probability):
+        """Random token ids with the verifier's arg-max planted on children, level by level (untimed)."""
+        torch = self.torch
+        n = len(parent)
+        depth = ssd_synth.tree_depths(parent)
+        out = []
+        for _ in range(sets):
+            tokens = ssd_synth.uniform_tokens(n, self.V, self.rng)
+            for lvl in range(1, int(depth.max()) + 1 if n > 1 else 0):
+                self.ctx.verify_tree(tokens, parent, self.kv, self.logits.data_ptr())
+                best = torch.argmax(self.logits[:n], dim=1).cpu().numpy()
+                for c in np.nonzero(depth == lvl)[0]:
+                    if self.rng.random() < probability:
+                        tokens[c] = int(best[parent[c]])
+            out.append(tokens)
+        return out
+
+    def time_steps(self, parent, token_sets, steps, warmup, draft=None, sampling=None, evict_l2=False):
+        """Runs warmup + steps full steps; device time of the whole loop and of every verify call."""
+        torch, ssd, ctx, kv = self.torch, self.ssd, self.ctx, self.kv
+        if evict_l2 and self.evict is None:
+            self.evict = torch.empty(256 * 1024 * 1024, dtype=torch.uint8, device="cuda")  # larger than the 126 MB L2
+
+        def one(i, ev=None):
+            tokens = token_sets[i % len(token_sets)]
+            if evict_l2:
+                self.evict.add_(1)
+            if ev is not None:
+                ev[0].record(self.stream)
+            ctx.verify_tree(tokens, parent, kv, self.logits.data_ptr())
+            if ev is not None:
+                ev[1].record(self.stream)
+            if sampling:
+                path, nxt = ctx.accept_tree(self.logits.data_ptr(), draft.data_ptr(), tokens, parent, mode=ssd.SSD_SAMPLING,
+                                            temperature=sampling[0], top_k=sampling[1], rng=self.srng)
+            else:
+                path, nxt = ctx.accept_tree(self.logits.data_ptr(), None, tokens, parent, mode=ssd.SSD_GREEDY, rng=self.srng)
+            ctx.kv_commit(kv, path)
+            kv.rollback(self.P)
+            return len(path)
+
+        for i in range(warmup):
+            one(i)
+        torch.cuda.synchronize()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        vev = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(steps)]
+        lengths = []
+        launches0 = ctx.kernel_launches()
+        t0 = time.perf_counter()
+        e0.record(self.stream)
+        for k in range(steps):
+            lengths.append(one(warmup + k, vev[k]))
+        e1.record(self.stream)
+        torch.cuda.synchronize()
+        wall = time.perf_counter() - t0
+        return {"dev_ms": e0.elapsed_time(e1), "wall_ms": wall * 1e3, "verify_us": [a.elapsed_time(b) * 1e3 for a, b in vev],
+                "lengths": lengths, "launches": ctx.kernel_launches() - launches0}
+
+    def kernel_timeline(self, parent, tokens):
+        """Per-kernel device time of one forward from the library's timeline (nanosecond timer stamps taken inside the
+        kernels): for every kernel the time from its dependencies being met to its latest CTA's end."""
+        ssd, ctx = self.ssd, self.ctx
+        ctx.set_tuning(ssd.SSD_TUNE_KERNEL_TRACE, 1)
+        for _ in range(3):
+            ctx.verify_tree(tokens, parent, self.kv, self.logits.data_ptr())
+        self.torch.cuda.synchronize()
+        t = ctx.phase_trace().astype(np.int64).reshape(-1, 8)
+        ctx.set_tuning(ssd.SSD_TUNE_KERNEL_TRACE, 0)
+        return t
+
+    def close(self):
+        self.kv.close()
+        self.ctx.close()
+
+
+def per_kernel_roofline(run: Runner, parent, tokens, peak_gbs):
+    """Achieved HBM GB/s of each projection kernel of a layer and of the LM head, from the device-side timeline."""
+    cfg = run.cfg
+    L, d, F, V = cfg["n_layer"], cfg["d_model"], cfg["d_ff"], cfg["vocab"]
+    t = run.kernel_timeline(parent, tokens)
+    setup = 3
+    per = (len(t) - setup - 2) // L
+    if per not in (5, 8) or len(t) != setup + per * L + 2:
+        return None
+    body = t[setup:setup + per * L].reshape(L, per, 8)
+    dur = (body[:, :, 6] - body[:, :, 1]) / 1e3  # dependencies met -> latest end, us
+    med = np.median(dur[2:], axis=0)
+    names = ["ln1", "qkv", "attention", "o_proj", "ln2", "fc", "gelu", "proj"] if per == 8 else ["qkv", "attention", "o_proj", "fc", "proj"]
+    weight_bytes = {"qkv": 2 * 3 * d * d, "o_proj": 2 * d * d, "fc": 2 * d * F, "proj": 2 * d * F}
+    out = {}
+    for name, us in zip(names, med):
+        e = {"us": float(us)}
+        if name in weight_bytes:
+            e["algorithmic_bytes"] = weight_bytes[name]
+            e["achieved_gbs"] = weight_bytes[name] / (us * 1e-6) / 1e9
+            e["frac"] = e["achieved_gbs"] / peak_gbs
+        out[name] = e
+    head_us = float(t[-1, 6] - t[-1, 1]) / 1e3
+    head_bytes = 2 * V * d + 4 * len(parent) * V
+    out["lm_head"] = {"us": head_us, "algorithmic_bytes": head_bytes, "achieved_gbs": head_bytes / (head_us * 1e-6) / 1e9,
+                      "frac": head_bytes / (head_us * 1e-6) / 1e9 / peak_gbs}
+    deps = body[:, 0, 1].astype(np.float64)
+    out["layer_us"] = float((deps[-1] - deps[2]) / (L - 3) / 1e3)
+    out["how"] = ("device timer stamps taken inside the kernels of one traced forward (dependencies met -> latest CTA end), "
+                  "median over layers; tracing itself slows the forward by a few percent")
+    return out
+
+
+def sweep_entry(label, cfg, n, P, res, peaks):
+    v = percentiles(res["verify_us"])
+    alg = ssd_synth.algorithmic_bytes(cfg, P, n)
+    fl = gemm_flops(cfg, n)
+    gbs = alg / (v["median"] * 1e-6) / 1e9
+    return {"workload": label, "n_nodes": n, "prefix": P, "verify_us": v, "step_us": res["dev_ms"] * 1e3 / len(res["verify_us"]),
+            "algorithmic_bytes": alg, "achieved_gbs": gbs, "frac_hbm_measured": gbs / peaks["hbm_gbs"], "frac_hbm_8TBs": gbs / NOMINAL_HBM_GBS,
+            "gemm_flops": fl, "frac_tensor_sustained": fl / (v["median"] * 1e-6) / 1e12 / peaks["bf16_tflops_sustained"],
+            "bound_us": {"hbm": alg / peaks["hbm_gbs"] / 1e3, "tensor": fl / peaks["bf16_tflops_sustained"] / 1e6},
+            "accepted_nodes_per_step": float(np.mean(res["lengths"]))}
+
+
+def run_sweep(args, local, peaks):
+    """The other configurations the benchmark is defined on, measured in the same process (one GPU only)."""
+    out = {}
+    steps, warm = max(10, min(args.steps, 30)), 3
+    # ---- GPT-2-small-shaped draft verified in the second stage: 512-token prefix, eight-node trigram tree
+    run = Runner("gpt2_small", 512, local, args.tune)
+    tokens, parent, rows = ssd_synth.trigram_tree(11, 22, 33, run.V)
+    warm_res = run.time_steps(parent, [tokens], steps, warm)
+    cold_res = run.time_steps(parent, [tokens], steps, warm, evict_l2=True)
+    e = sweep_entry("gpt2_small stage-two verify, trigram tree", run.cfg, len(parent), 512, warm_res, peaks)
+    e["verify_us_l2_evicted"] = percentiles(cold_res["verify_us"])
+    e["l2_note"] = "268 MB of algorithmic bytes against a 126 MB L2: 'evicted' writes a 256 MB buffer between steps"
+    out["config3"] = e
+    run.close()
+    del run
+    # ---- GPT-2-XL-shaped model: tree sizes 8..256, random parents with depth <= 8
+    run = Runner("gpt2_xl", 512, local, args.tune)
+    rows_xl = []
+    for n in (8, 16, 32, 64, 128, 256):
+        parent = ssd_synth.tree_random(n, 8, run.rng)
+        toks = [ssd_synth.uniform_tokens(n, run.V, run.rng) for _ in range(4)]
+        rows_xl.append(sweep_entry("gpt2_xl verify, random tree of depth <= 8", run.cfg, n, 512, run.time_steps(parent, toks, steps, warm), peaks))
+    cfg = run.cfg
+    run.close()
+    del run
+    # the tree size at which the tensor bound (at the sustained bf16 peak) overtakes the HBM bound (at the measured copy bandwidth)
+    cross = None
+    for n in range(1, 1025):
+        if gemm_flops(cfg, n) / (peaks["bf16_tflops_sustained"] * 1e12) > ssd_synth.algorithmic_bytes(cfg, 512, n) / (peaks["hbm_gbs"] * 1e9):
+            cross = n
+            break
+    t = [r["verify_us"]["median"] for r in rows_xl]
+    out["config5"] = {"rows": rows_xl, "crossover_nodes_of_the_bounds": cross,
+                      "measured_us_per_node_beyond_64": (t[5] - t[3]) / (256 - 64),
+                      "note": "below the crossover the forward can at best run at the HBM bound, above it at the tensor bound; measured times "
+                              "are several times either bound (a chain of dependent kernels), and grow roughly linearly in the tree size from 64 nodes on"}
+    return out
+
+
 def run_gpu(args):
     import torch
-    import paper_2308_04623_b200 as ssd
 
     rank = int(os.environ.get("RANK", "0"))
     local = int(os.environ.get("LOCAL_RANK", "0"))
@@ -194,45 +426,11 @@ def run_gpu(args):
         import torch.distributed as dist
         dist.init_process_group("nccl", device_id=torch.device("cuda", local))
     cfg, parent = workload(args)
-    V, n, P = cfg["vocab"], len(parent), args.prefix
-    rng = np.random.default_rng(1002 + rank)
-    weights = ssd_synth.make_weights(cfg, seed=0)
-    stream = torch.cuda.current_stream()
-    ctx = ssd.Context(cfg, device=local, stream=stream.cuda_stream)
-    ctx.load_weights(ssd_synth.bf16_bits(weights) if cfg["dtype"] == "bf16" else weights)
-    for spec in args.tune:
-        knob, value = spec.split("=")
-        ctx.set_tuning(int(knob), int(value))
-    kv = ctx.new_kv()
-    logits = torch.empty((max(n, 256), V), dtype=torch.float32, device="cuda")
-    # prefix through hot-path calls only: chain trees, every node committed
-    prefix = ssd_synth.uniform_tokens(P, V, rng)
-    for s in range(0, P, 256):
-        t = prefix[s:s + 256]
-        ctx.verify_tree(t, ssd_synth.tree_chain(len(t)), kv, logits.data_ptr())
-        ctx.kv_commit(kv, np.arange(len(t), dtype=np.int32))
-    total = args.warmup + args.steps
-    toks = [ssd_synth.uniform_tokens(n, V, rng) for _ in range(total + 4)]
-    srng = ssd.binding.ssd_rng(1, 0)
-    sampling = args.accept == "sampling"
-    draft = None
-    if sampling:  # one proposal row per node, resident on the device like the logits
-        draft = torch.from_numpy(ssd_synth.draft_rows_gamma(n, V, rng)).cuda()
-
-    def one_step(i, ev=None):
-        if ev is not None:
-            ev[0].record(stream)
-        ctx.verify_tree(toks[i], parent, kv, logits.data_ptr())
-        if ev is not None:
-            ev[1].record(stream)
-        if sampling:
-            path, nxt = ctx.accept_tree(logits.data_ptr(), draft.data_ptr(), toks[i], parent, mode=ssd.SSD_SAMPLING,
-                                        temperature=args.temperature, top_k=args.top_k, rng=srng)
-        else:
-            path, nxt = ctx.accept_tree(logits.data_ptr(), None, toks[i], parent, mode=ssd.SSD_GREEDY, rng=srng)
-        ctx.kv_commit(kv, path)
-        kv.rollback(P)
-        return len(path)
+    n, P = len(parent), args.prefix
+    run = Runner(args.model, P, local, args.tune, rng_seed=1002 + rank)
+    sampling = (args.temperature, args.top_k) if args.accept == "sampling" else None
+    draft = torch.from_numpy(ssd_synth.draft_rows_gamma(n, run.V, run.rng)).cuda() if sampling else None
+    token_sets = run.planted_tokens(parent, 8, PLANT_PROBABILITY)
 
     def barrier():
         if world > 1:
@@ -240,70 +438,69 @@ def run_gpu(args):
             dist.barrier()
         torch.cuda.synchronize()
 
-    for i in range(args.warmup):
-        one_step(i)
-    # ---- timed region 1: device time over exactly K steps (events on the library's stream)
+    run.time_steps(parent, token_sets, 1, args.warmup, draft, sampling)  # warm-up
     sampler = ClockSampler(local)
     if rank == 0:
         sampler.start()
     barrier()
-    launches0 = ctx.kernel_launches()
-    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    vev = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(args.steps)]
-    accepted = 0
-    t_wall0 = time.perf_counter()
-    e0.record(stream)
-    for k in range(args.steps):
-        accepted += one_step(args.warmup + k, vev[k])
-    e1.record(stream)
+    res = run.time_steps(parent, token_sets, args.steps, 0, draft, sampling)  # ---- the timed region: exactly K steps
     barrier()
-    wall = time.perf_counter() - t_wall0
-    launches = ctx.kernel_launches() - launches0
     clocks = sampler.stop() if rank == 0 else {}
-    dev_ms = e0.elapsed_time(e1)
-    verify_ms = float(np.mean([a.elapsed_time(b) for a, b in vev]))
-    status = ctx.device_status()
-    dev_ms, wall_ms, verify_ms = max_over_ranks([dev_ms, wall * 1e3, verify_ms])
+    status = run.ctx.device_status()
+    v = percentiles(res["verify_us"])
+    dev_ms, wall_ms, verify_med = max_over_ranks([res["dev_ms"], res["wall_ms"], v["median"]])
     if rank != 0:
+        run.close()
         return
     ms_per_step = dev_ms / args.steps
     peaks, peak_kind = measured_peaks()
     alg_bytes = ssd_synth.algorithmic_bytes(cfg, P, n)
-    achieved = alg_bytes / (verify_ms * 1e-3) / 1e9
+    achieved = alg_bytes / (verify_med * 1e-6) / 1e9
+    lengths = np.asarray(res["lengths"])
+    hist = {str(k): int((lengths == k).sum()) for k in sorted(set(lengths.tolist()))}
     line = {
         "metric": METRIC, "value": replica_value(ms_per_step, world), "unit": UNIT, "n_gpus": world, "steps": args.steps,
         "warmup": args.warmup, "ms_per_step": ms_per_step, "higher_is_better": False, "scaling": "weak", "vs_baseline": None,
         "dtype": "bf16" if cfg["dtype"] == "bf16" else "f32", "data": "synthetic",
         "config": {"workload": "%s verify n=%d prefix=%d, %s accept, commit" % (
                        args.model, n, P, ("sampling (T=%g, top-k=%d)" % (args.temperature, args.top_k)) if sampling else "greedy"),
-                   "tree": "branching %s BFS truncated at %d" % (list(tree_rule(n)), n), "l2": "inputs larger than L2 (%.0f MB of weights per step)"
-                   % (alg_bytes / 1e6), "replicas": world, "aggregate": "per-replica step time / n_gpus",
-                   "accepted_tokens_per_step": accepted / args.steps},
-        "verify_us": verify_ms * 1e3, "steps_per_s": world * 1e3 / ms_per_step,
-        # every accepted node of the path (the root included) emits one token: tokens[path[1:]] and the extra one
-        "emitted_tokens_per_s": world * 1e3 / ms_per_step * accepted / args.steps,
-        "roofline": {"bound": "hbm", "kernel": "ssd_verify_tree (all launches of one forward)", "achieved": achieved,
-                     "peak": peaks["hbm_gbs"], "peak_kind": "of " + peak_kind, "unit": "GB/s", "frac": achieved / peaks["hbm_gbs"],
-                     "frac_of_nominal_8TBs": achieved / NOMINAL_HBM_GBS, "algorithmic_bytes": alg_bytes, "traffic": NCU_TRAFFIC_BYTES.get((args.model, n, P))},
+                   "tree": "branching %s BFS truncated at %d" % (list(tree_rule(n)), n),
+                   "tokens": "uniform ids, the verifier's arg-max planted on each child with probability %g" % PLANT_PROBABILITY,
+                   "l2": "inputs larger than L2 (%.0f MB of weights per step)" % (alg_bytes / 1e6), "replicas": world,
+                   "aggregate": "per-replica step time / n_gpus", "accepted_nodes_per_step": float(lengths.mean()),
+                   "accepted_path_length_histogram": hist},
+        "verify_us": verify_med, "verify_us_percentiles": v, "steps_per_s": world * 1e3 / ms_per_step,
+        # every node of the accepted path (the root included) emits one token: tokens[path[1:]] and the extra one
+        "emitted_tokens_per_s": world * 1e3 / ms_per_step * float(lengths.mean()),
+        "roofline": {"bound": "hbm", "kernel": "ssd_verify_tree (all launches of one forward; per-kernel figures under roofline_per_kernel)",
+                     "achieved": achieved, "peak": peaks["hbm_gbs"], "peak_kind": "of " + peak_kind, "unit": "GB/s",
+                     "frac": achieved / peaks["hbm_gbs"], "frac_of_nominal_8TBs": achieved / NOMINAL_HBM_GBS, "algorithmic_bytes": alg_bytes,
+                     "traffic": NCU_TRAFFIC_BYTES.get((args.model, n, P))},
         "e2e": {"value": wall_ms * 1e3 / args.steps / world, "unit": UNIT, "h2d_bytes_per_step": 4 * n * 4 + 4 * n,
                 "d2h_bytes_per_step": 4 * (n + 4)},
-        "gpu_launches": int(launches), "clocks": clocks, "device_status": status,
+        "gpu_launches": int(res["launches"]), "clocks": clocks, "device_status": status,
     }
+    if world == 1:
+        line["roofline_per_kernel"] = per_kernel_roofline(run, parent, token_sets[0], peaks["hbm_gbs"])
+    weights = run.weights
+    run.close()
+    del run
+    if world == 1 and not args.no_sweep:
+        sweep = {}
+        for nn in (16, 64):
+            r2 = Runner(args.model, P, local, args.tune)
+            par = ssd_synth.tree_branching(nn, tree_rule(nn))
+            toks = r2.planted_tokens(par, 4, PLANT_PROBABILITY)
+            sweep["n%d" % nn] = sweep_entry("%s verify" % args.model, cfg, nn, P, r2.time_steps(par, toks, max(10, min(args.steps, 30)), 3), peaks)
+            r2.close()
+            del r2
+        sweep.update(run_sweep(args, local, peaks))
+        line["sweep"] = sweep
     if world == 1 and not args.no_cpu_baseline:
-        sn, sp = min(args.ref_nodes, n), args.ref_prefix
-        step = oracle_sample_step(cfg, weights, parent, sn, sp, rng)
-        t0 = time.perf_counter()
-        reps = 0
-        while reps < 2 or (time.perf_counter() - t0 < 10.0 and reps < 20):
-            step()
-            reps += 1
-        cpu_us = (time.perf_counter() - t0) / reps * 1e6 * (n / sn)
-        line["cpu_baseline"] = {"value": cpu_us, "unit": UNIT, "cores": omp_threads(), "kind": "oracle",
-                                "sample": "%d oracle steps on the first %d nodes of the tree at prefix %d, time scaled by %g"
-                                % (reps, sn, sp, n / sn)}
+        times = oracle_steps(cfg, weights, parent, P, np.random.default_rng(7), 3, 0, 60.0)
+        line["cpu_baseline"] = {"value": float(np.median(times)) * 1e6, "unit": UNIT, "cores": omp_threads(), "kind": "oracle",
+                                "sample": "%d full oracle steps (the whole %d-node tree at prefix %d), median" % (len(times), n, P)}
     print(json.dumps(line), flush=True)
-    kv.close()
-    ctx.close()
 
 
 def main():
@@ -315,10 +512,9 @@ def main():
     ap.add_argument("--model", default="gpt2_large")
     ap.add_argument("--nodes", type=int, default=32)
     ap.add_argument("--prefix", type=int, default=256)
-    ap.add_argument("--ref-nodes", type=int, default=8)
-    ap.add_argument("--ref-prefix", type=int, default=32)
     ap.add_argument("--ref-budget-s", type=float, default=150.0)
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-sweep", action="store_true", help="skip the other configurations (16 / 64 nodes, draft model, XL sweep)")
     ap.add_argument("--tune", action="append", default=[], help="knob=value for ssd_set_tuning (experiments)")
     ap.add_argument("--accept", default="greedy", choices=["greedy", "sampling"],
                     help="acceptance rule of the step (the metric's workload is greedy; sampling draws draft rows from a Dirichlet)")
@@ -326,6 +522,8 @@ def main():
     ap.add_argument("--temperature", type=float, default=1.0)
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "ssd" else args.warmup
+    if args.gpus > 1 and "WORLD_SIZE" not in os.environ:
+        sys.exit(spawn_replicas(args.gpus, sys.argv[1:]))  # one process per GPU; under torchrun the ranks exist already
     if args.impl == "reference":
         run_reference(args)
     else:
