@@ -233,6 +233,18 @@ int ssd_get_phase_trace(ssd_ctx *ctx, uint64_t *out_ns, int32_t capacity, int32_
 const char *ssd_strerror(int status);
 /* Device-side status word of the last launches (0 = clean; non-zero: a bounded wait gave up). */
 int ssd_last_device_status(ssd_ctx *ctx, int32_t *word);
+/*
+ * Failure handling of the device-side waits.  Every wait inside the kernels (on an mbarrier that a copy, an MMA or
+ * another warp completes) is bounded; when one expires the kernel records a non-zero word, leaves its loops, frees
+ * its tensor memory and returns, and every later projection kernel of the context becomes a no-op while the word is
+ * set.  ssd_accept_tree - the step's one synchronisation point - reads the word with its results and returns
+ * SSD_ERR_TIMEOUT when it is set.  ssd_reset_device_status clears the word (waits for the stream); the context is
+ * then usable again.  ssd_debug_expire_wait is a test hook: it enqueues a tiny kernel in which one warp waits
+ * `limit_us` microseconds on an mbarrier at which nothing arrives - nothing else is in flight - and records the
+ * word 0xE00, so that the whole failure path can be exercised without making a production kernel time out.
+ */
+int ssd_reset_device_status(ssd_ctx *ctx);
+int ssd_debug_expire_wait(ssd_ctx *ctx, int32_t limit_us);
 /* cudaError_t value of the last failed CUDA call on this context (0 if none). */
 int ssd_last_cuda_error(const ssd_ctx *ctx);
 /* Line of the library's API source file where that call failed (diagnostic aid; 0 if none). */

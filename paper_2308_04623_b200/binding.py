@@ -19,7 +19,7 @@ SSD_TUNE_CLUSTER_QKV, SSD_TUNE_CLUSTER_O, SSD_TUNE_CLUSTER_FC, SSD_TUNE_CLUSTER_
 # every symbol include/ssd.h declares
 EXPORTS = ("ssd_create", "ssd_load_weights", "ssd_kv_create", "ssd_kv_reset", "ssd_kv_len", "ssd_kv_rollback",
            "ssd_kv_destroy", "ssd_verify_tree", "ssd_accept_tree", "ssd_kv_commit", "ssd_kv_read", "ssd_strerror",
-           "ssd_last_device_status", "ssd_last_cuda_error", "ssd_last_cuda_error_line", "ssd_kernel_launches", "ssd_set_tuning", "ssd_get_phase_trace", "ssd_accept_tree_noalloc", "ssd_destroy")
+           "ssd_last_device_status", "ssd_reset_device_status", "ssd_debug_expire_wait", "ssd_last_cuda_error", "ssd_last_cuda_error_line", "ssd_kernel_launches", "ssd_set_tuning", "ssd_get_phase_trace", "ssd_accept_tree_noalloc", "ssd_destroy")
 
 
 class ssd_config(C.Structure):
@@ -80,6 +80,8 @@ def lib():
         L.ssd_last_cuda_error.argtypes = [_VP]
         L.ssd_last_cuda_error_line.argtypes = [_VP]
         L.ssd_kernel_launches.argtypes = [_VP, C.POINTER(C.c_int64)]
+        L.ssd_reset_device_status.argtypes = [_VP]
+        L.ssd_debug_expire_wait.argtypes = [_VP, C.c_int32]
         L.ssd_set_tuning.argtypes = [_VP, C.c_int32, C.c_int32]
         L.ssd_get_phase_trace.argtypes = [_VP, _VP, C.c_int32, C.POINTER(C.c_int32)]
         L.ssd_destroy.argtypes = [_VP]
@@ -189,6 +191,12 @@ class Context:
         w = C.c_int32(0)
         self._chk(lib().ssd_last_device_status(self.h, C.byref(w)))
         return w.value
+
+    def reset_device_status(self) -> None:
+        self._chk(lib().ssd_reset_device_status(self.h))
+
+    def debug_expire_wait(self, limit_us: int = 10) -> None:
+        self._chk(lib().ssd_debug_expire_wait(self.h, int(limit_us)))
 
     def kernel_launches(self) -> int:
         c = C.c_int64(0)

@@ -9,6 +9,7 @@
 #include <cstring>
 #include <mutex>
 
+#include "sm100_ptx.cuh"
 #include "ssd_internal.h"
 
 namespace {
@@ -69,9 +70,11 @@ __global__ void __launch_bounds__(256) row_argmax_kernel(const float *__restrict
 // The walk; a row's arg-max is the best of its `parts` parts (the parts are in index order, so the first one that
 // attains the maximum holds the lowest index).  `result` may be pinned host memory.
 __global__ void greedy_walk_kernel(NodeList tokens, NodeList parent, int n, int parts, const float *__restrict__ part_val,
-                                   const int32_t *__restrict__ part_arg, const int32_t *__restrict__ part_bad, int32_t *__restrict__ result) {
+                                   const int32_t *__restrict__ part_arg, const int32_t *__restrict__ part_bad, int32_t *__restrict__ result,
+                                   const int32_t *__restrict__ dev_status) {
     if (threadIdx.x != 0) return;
     int cur = 0, np = 1;
+    result[3] = dev_status ? *dev_status : 0; // the forward's error word rides along with the walk's few result words
     result[4] = 0;
     for (;;) {
         float best = -INFINITY;
@@ -346,11 +349,11 @@ __device__ int node_decide(double *__restrict__ r, int cnt, const int32_t *__res
 __global__ void __launch_bounds__(ACC_THREADS) sample_walk_kernel(const float *__restrict__ logits, const float *__restrict__ draft,
                                                                   NodeList tokens, NodeList parent, int n, int V, double temperature,
                                                                   int top_k, uint64_t seed, uint64_t step, double *__restrict__ r,
-                                                                  int32_t *__restrict__ result) {
+                                                                  int32_t *__restrict__ result, const int32_t *__restrict__ dev_status) {
     __shared__ BlockScratch s;
     const int tid = threadIdx.x;
     int cur = 0, np = 1;
-    if (tid == 0) result[4] = 0;
+    if (tid == 0) { result[3] = dev_status ? *dev_status : 0; result[4] = 0; }
     for (;;) {
         // a visited row must be finite
         if (row_law(logits + (size_t)cur * V, V, temperature, top_k, r, s)) {
@@ -389,9 +392,11 @@ __global__ void __launch_bounds__(ACC_THREADS) node_decide_kernel(const float *_
 }
 
 // Follows next[] from the root.  `result` may be pinned host memory.
-__global__ void chain_walk_kernel(const int32_t *__restrict__ next, const int32_t *__restrict__ bonus, int n, int32_t *__restrict__ result) {
+__global__ void chain_walk_kernel(const int32_t *__restrict__ next, const int32_t *__restrict__ bonus, int n, int32_t *__restrict__ result,
+                                  const int32_t *__restrict__ dev_status) {
     if (threadIdx.x != 0) return;
     int cur = 0, np = 1;
+    result[3] = dev_status ? *dev_status : 0;
     result[4] = 0;
     for (;;) {
         const int c = next[cur];
@@ -409,7 +414,7 @@ cudaError_t launch_accept(const float *logits, const float *draft_probs, const N
     if (mode == SSD_GREEDY) {
         const int parts = sc.arg_parts > 0 ? sc.arg_parts : 1;
         row_argmax_kernel<<<dim3(n, parts), 256, 0, s>>>(logits, vocab, sc.row_val, sc.row_arg, sc.row_bad);
-        greedy_walk_kernel<<<1, 32, 0, s>>>(tokens, parent, n, parts, sc.row_val, sc.row_arg, sc.row_bad, sc.result);
+        greedy_walk_kernel<<<1, 32, 0, s>>>(tokens, parent, n, parts, sc.row_val, sc.row_arg, sc.row_bad, sc.result, sc.dev_status);
         *launches += 2;
     } else {
         double *rows = (sc.rows && sc.rows_cap >= n && n > 1) ? sc.rows : nullptr;
@@ -419,14 +424,30 @@ cudaError_t launch_accept(const float *logits, const float *draft_probs, const N
             row_law_kernel<<<n, ACC_THREADS, 0, s>>>(logits, vocab, (double)temperature, top_k, rows, sc.row_bad, sc.sup_idx, sc.sup_cnt);
             node_decide_kernel<<<n, ACC_THREADS, 0, s>>>(draft_probs, tokens, parent, n, vocab, seed, step, rows, sc.row_bad, sc.sup_idx, sc.sup_cnt,
                                                          next, bonus);
-            chain_walk_kernel<<<1, 32, 0, s>>>(next, bonus, n, sc.result);
+            chain_walk_kernel<<<1, 32, 0, s>>>(next, bonus, n, sc.result, sc.dev_status);
             *launches += 3;
         } else {
             sample_walk_kernel<<<1, ACC_THREADS, 0, s>>>(logits, draft_probs, tokens, parent, n, vocab, (double)temperature, top_k, seed, step,
-                                                         sc.r, sc.result);
+                                                         sc.r, sc.result, sc.dev_status);
             *launches += 1;
         }
     }
+    return cudaGetLastError();
+}
+
+// ---------------------------------------------------------------------------------------------
+// A wait that runs out, for testing the failure path without touching the production kernels: one warp waits, with
+// the same bounded wait the projection kernels use, on an mbarrier at which nothing ever arrives (no copy, no MMA and
+// no tensor memory is in flight), records the error word when the limit expires and returns.
+// ---------------------------------------------------------------------------------------------
+__global__ void expired_wait_kernel(int32_t *status, long long limit_cycles) {
+    __shared__ uint64_t bar;
+    if (threadIdx.x == 0) { ptx::mbar_init(&bar, 1); ptx::fence_mbar_init(); }
+    __syncwarp();
+    if (threadIdx.x == 0 && !ptx::mbar_wait_bounded(&bar, 0, limit_cycles)) atomicExch(status, 0xE00);
+}
+cudaError_t launch_expired_wait(int32_t *status, long long limit_cycles, cudaStream_t s) {
+    expired_wait_kernel<<<1, 32, 0, s>>>(status, limit_cycles);
     return cudaGetLastError();
 }
 
@@ -470,6 +491,7 @@ cudaError_t noalloc_setup(int device, AcceptScratch *out) {
         slot.sc.row_arg = (int32_t *)arg;
         slot.sc.row_bad = (int32_t *)bad;
         slot.sc.result = (int32_t *)res;
+        slot.sc.dev_status = nullptr;
         slot.ready = true;
     }
     *out = slot.sc;

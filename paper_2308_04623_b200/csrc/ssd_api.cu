@@ -365,6 +365,7 @@ int ssd_create(const ssd_config *cfg, int device, void *cuda_stream, ssd_ctx **o
     A(&ctx->meta.anc, n * SSD_ANC_WORDS); A(&ctx->meta.child_off, n + 1); A(&ctx->meta.child, n);
     A(&ctx->x, n * d); A(&ctx->a, n * d); A(&ctx->qkv, n * 3 * d); A(&ctx->o, n * d); A(&ctx->h, n * (size_t)cfg->d_ff);
     ctx->acc.arg_parts = 4;
+    ctx->acc.dev_status = nullptr;
     A(&ctx->acc.r, (size_t)cfg->vocab); A(&ctx->acc.row_val, 4 * n); A(&ctx->acc.row_arg, 4 * n); A(&ctx->acc.row_bad, 4 * n); A(&ctx->acc.result, n + 4);
     A(&ctx->d_status, 1);
     A(&ctx->d_info, 1);
@@ -638,6 +639,7 @@ int ssd_accept_tree(ssd_ctx *ctx, const float *logits, const float *draft_probs,
     int launched = 0;
     AcceptScratch sc = ctx->acc;
     sc.result = ctx->h_result; // the walk writes its few words straight into the pinned host buffer: no copy to enqueue and wait for
+    sc.dev_status = ctx->d_status;
     ctx->h_result[0] = 0;
     CU(launch_accept(logits, draft_probs, tk, pr, n, c.vocab, sampling->mode, sampling->temperature, sampling->top_k, rng_state->seed,
                      rng_state->step, sc, ctx->stream, &launched));
@@ -649,6 +651,9 @@ int ssd_accept_tree(ssd_ctx *ctx, const float *logits, const float *draft_probs,
     *n_path_out = np;
     *next_token_out = ctx->h_result[1];
     memcpy(path_out, ctx->h_result + 4, sizeof(int32_t) * np);
+    // A bounded wait of one of the forward's kernels expired (the word stays set, and later forwards are no-ops, until
+    // ssd_reset_device_status): the logits this walk read are not to be trusted.
+    if (ctx->h_result[3] != 0) return SSD_ERR_TIMEOUT;
     return ctx->h_result[2];
 }
 
@@ -696,6 +701,22 @@ int ssd_last_device_status(ssd_ctx *ctx, int32_t *word) {
     if (!g.ok) return SSD_ERR_CUDA;
     CU(cudaMemcpyAsync(word, ctx->d_status, sizeof(int32_t), cudaMemcpyDeviceToHost, ctx->stream));
     CU(cudaStreamSynchronize(ctx->stream));
+    return SSD_OK;
+}
+int ssd_reset_device_status(ssd_ctx *ctx) {
+    if (!ctx) return SSD_ERR_BAD_ARG;
+    DeviceGuard g(ctx->device);
+    if (!g.ok) return SSD_ERR_CUDA;
+    CU(cudaMemsetAsync(ctx->d_status, 0, sizeof(int32_t), ctx->stream));
+    CU(cudaStreamSynchronize(ctx->stream));
+    return SSD_OK;
+}
+int ssd_debug_expire_wait(ssd_ctx *ctx, int32_t limit_us) {
+    if (!ctx || limit_us < 1 || limit_us > 1000000) return SSD_ERR_BAD_ARG;
+    DeviceGuard g(ctx->device);
+    if (!g.ok) return SSD_ERR_CUDA;
+    CU(launch_expired_wait(ctx->d_status, (long long)limit_us * 2000ll, ctx->stream)); // ~2 GHz SM clock
+    ctx->launches += 1;
     return SSD_OK;
 }
 int ssd_set_tuning(ssd_ctx *ctx, int32_t knob, int32_t value) {

@@ -139,8 +139,10 @@ struct AcceptScratch {
     float *row_val;     // [max_nodes * parts] per-part row maximum (greedy)
     int32_t *row_arg;   // [max_nodes * parts] per-part arg-max (greedy)
     int32_t *row_bad;   // [max_nodes * parts] 1 if the part holds a non-finite value (sampling: [max_nodes], per row)
-    int32_t *result;    // [max_nodes + 4]: n_path, next_token, status, pad, path[...]
+    int32_t *result;    // [max_nodes + 4]: n_path, next_token, status, device error word, path[...]
+    const int32_t *dev_status; // the forward's device error word (copied into result[3] by the walk) or null
 };
+cudaError_t launch_expired_wait(int32_t *status, long long limit_cycles, cudaStream_t s);
 cudaError_t launch_accept(const float *logits, const float *draft_probs, const NodeList &tokens, const NodeList &parent, int n,
                           int vocab, int mode, float temperature, int top_k, uint64_t seed, uint64_t step,
                           const AcceptScratch &sc, cudaStream_t s, int *launches);

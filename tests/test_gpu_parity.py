@@ -573,3 +573,38 @@ def test_kernel_timeline_has_eight_ordered_stamps_per_launch(util, ssd):
         assert p.ctx.device_status() == 0
     finally:
         p.close()
+
+
+# --------------------------------------------------------------------------- failure path (a wait that runs out, made safely)
+def test_expired_device_wait_surfaces_as_timeout_and_can_be_reset(util, ssd):
+    """A bounded device-side wait that expires must reach the caller: the test hook makes one warp wait 10 us on an
+    mbarrier nobody arrives at (nothing else in flight), which records the error word.  The next accept returns
+    SSD_ERR_TIMEOUT, a verify enqueued while the word is set leaves its projections undone, and after a reset the
+    context computes the right logits again."""
+    p = util.Pair("tiny_bf16", seed=5, qk_gain=3.0)
+    try:
+        rng = np.random.default_rng(21)
+        p.prefill(ssd_synth.uniform_tokens(19, p.V, rng), chunk=16)
+        parent = ssd_synth.tree_random(12, 4, rng)
+        tokens = ssd_synth.uniform_tokens(12, p.V, rng)
+        good, want, buf = p.verify(tokens, parent)
+        assert np.abs(good - want).max() <= TOL_BF16 and p.ctx.device_status() == 0
+        p.ctx.debug_expire_wait(10)
+        assert p.ctx.device_status() == 0xE00
+        with pytest.raises(ssd.SsdError) as e:
+            p.ctx.accept_tree(buf.data_ptr(), None, tokens, parent)
+        assert e.value.code == ssd.SSD_ERR_TIMEOUT
+        stale = torch.full((12, p.V), 7.0, dtype=torch.float32, device="cuda")
+        p.ctx.verify_tree(tokens, parent, p.kv, stale.data_ptr())   # projections are no-ops while the word is set
+        torch.cuda.synchronize()
+        assert float(stale.abs().max()) == 0.0                      # cleared at the start of the forward, never accumulated into
+        assert p.ctx.device_status() == 0xE00
+        p.ctx.reset_device_status()
+        assert p.ctx.device_status() == 0
+        again, _, buf = p.verify(tokens, parent)
+        assert np.abs(again - want).max() <= TOL_BF16
+        path, nxt = p.ctx.accept_tree(buf.data_ptr(), None, tokens, parent)
+        opath, onxt, _ = ssd_oracle.accept_tree(again.astype(np.float32), None, tokens, parent, mode=0)
+        assert (path, nxt) == (opath, onxt)
+    finally:
+        p.close()
