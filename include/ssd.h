@@ -254,6 +254,32 @@ int ssd_kernel_launches(const ssd_ctx *ctx, int64_t *count);
 
 void ssd_destroy(ssd_ctx *ctx);
 
+/*
+ * The lowest speculation stage: a Katz back-off trigram model (Section 4 names it as the model that proposes tokens
+ * for the small draft; Section 3.2 is the staging; the closing list of Section 4 asks for such proposers to answer
+ * in under 10 microseconds).  The paper gives no formula; the reading: counts over a token stream, absolute discount
+ * 0.5 at the trigram and bigram levels, back-off weights that make every level sum to one, a context never seen backs
+ * off entirely, and a context's proposals are its four most probable next tokens (ties towards the lower id).
+ *
+ * ssd_trigram_build    counts `stream_tokens` (host, n_tokens >= 3 ids in [0, vocab)) and builds the device tables (the
+ *                      answers of every context the stream contains); the handle owns them.  BAD_ARG, NOMEM, CUDA.
+ * ssd_trigram_lookup   contexts (host [m][2]: the two preceding tokens, m <= 4096) -> the four best next tokens and their
+ *                      probabilities (host [m][4] each).  Waits for the stream.
+ * ssd_trigram_propose  fills a proposal tree on the device: node 0 holds `root`, which `prev1` precedes; the children of a
+ *                      node, in index order, receive the best continuations of (the token before the node, the node's
+ *                      token).  parent_idx as in ssd_verify_tree, at most four children per node (else INVALID_TREE).
+ *                      tokens_out / probs_out: host [n_nodes] (probs_out[0] = 0).  One warp, four dependent table
+ *                      look-ups for the eight-node tree of the stage-two configuration.  Waits for the stream.
+ * ssd_trigram_contexts number of distinct two-token contexts in the table.
+ */
+typedef struct ssd_trigram ssd_trigram;
+int ssd_trigram_build(const int32_t *stream_tokens, int64_t n_tokens, int32_t vocab, int device, void *cuda_stream, ssd_trigram **out);
+int ssd_trigram_lookup(ssd_trigram *t, const int32_t *contexts, int32_t m, int32_t *tokens_out, float *probs_out);
+int ssd_trigram_propose(ssd_trigram *t, int32_t prev1, int32_t root, const int32_t *parent_idx, int32_t n_nodes, int32_t *tokens_out,
+                        float *probs_out);
+int ssd_trigram_contexts(const ssd_trigram *t, int64_t *count);
+void ssd_trigram_destroy(ssd_trigram *t);
+
 #ifdef __cplusplus
 }
 #endif

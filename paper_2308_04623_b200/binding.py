@@ -19,7 +19,8 @@ SSD_TUNE_CLUSTER_QKV, SSD_TUNE_CLUSTER_O, SSD_TUNE_CLUSTER_FC, SSD_TUNE_CLUSTER_
 # every symbol include/ssd.h declares
 EXPORTS = ("ssd_create", "ssd_load_weights", "ssd_kv_create", "ssd_kv_reset", "ssd_kv_len", "ssd_kv_rollback",
            "ssd_kv_destroy", "ssd_verify_tree", "ssd_accept_tree", "ssd_kv_commit", "ssd_kv_read", "ssd_strerror",
-           "ssd_last_device_status", "ssd_reset_device_status", "ssd_debug_expire_wait", "ssd_last_cuda_error", "ssd_last_cuda_error_line", "ssd_kernel_launches", "ssd_set_tuning", "ssd_get_phase_trace", "ssd_accept_tree_noalloc", "ssd_destroy")
+           "ssd_last_device_status", "ssd_reset_device_status", "ssd_debug_expire_wait", "ssd_last_cuda_error", "ssd_last_cuda_error_line", "ssd_kernel_launches", "ssd_set_tuning", "ssd_get_phase_trace", "ssd_accept_tree_noalloc", "ssd_destroy",
+           "ssd_trigram_build", "ssd_trigram_lookup", "ssd_trigram_propose", "ssd_trigram_contexts", "ssd_trigram_destroy")
 
 
 class ssd_config(C.Structure):
@@ -86,6 +87,12 @@ def lib():
         L.ssd_get_phase_trace.argtypes = [_VP, _VP, C.c_int32, C.POINTER(C.c_int32)]
         L.ssd_destroy.argtypes = [_VP]
         L.ssd_destroy.restype = None
+        L.ssd_trigram_build.argtypes = [_VP, C.c_int64, C.c_int32, C.c_int, _VP, C.POINTER(_VP)]
+        L.ssd_trigram_lookup.argtypes = [_VP, _VP, C.c_int32, _VP, _VP]
+        L.ssd_trigram_propose.argtypes = [_VP, C.c_int32, C.c_int32, _VP, C.c_int32, _VP, _VP]
+        L.ssd_trigram_contexts.argtypes = [_VP, C.POINTER(C.c_int64)]
+        L.ssd_trigram_destroy.argtypes = [_VP]
+        L.ssd_trigram_destroy.restype = None
         _lib = L
     return _lib
 
@@ -231,3 +238,46 @@ class KV:
 
     def rollback(self, n: int):
         self.ctx._chk(lib().ssd_kv_rollback(self.h, n))
+
+
+class Trigram:
+    """Handle of a Katz back-off trigram table on the device (argument marshalling only)."""
+
+    def __init__(self, stream_tokens, vocab: int, device: int = 0, stream: int = 0):
+        toks = np.ascontiguousarray(stream_tokens, dtype=np.int32)
+        h = _VP()
+        rc = lib().ssd_trigram_build(toks.ctypes.data, len(toks), int(vocab), int(device), _VP(stream), C.byref(h))
+        if rc != SSD_OK:
+            raise SsdError(rc)
+        self.h, self.vocab = h, int(vocab)
+
+    def lookup(self, contexts):
+        """contexts: [m, 2] preceding token pairs -> (tokens int32 [m, 4], probabilities float32 [m, 4])."""
+        ctx = np.ascontiguousarray(contexts, dtype=np.int32).reshape(-1, 2)
+        tok = np.zeros((len(ctx), 4), dtype=np.int32)
+        pr = np.zeros((len(ctx), 4), dtype=np.float32)
+        rc = lib().ssd_trigram_lookup(self.h, ctx.ctypes.data, len(ctx), tok.ctypes.data, pr.ctypes.data)
+        if rc != SSD_OK:
+            raise SsdError(rc)
+        return tok, pr
+
+    def propose(self, prev1: int, root: int, parent_idx):
+        par = np.ascontiguousarray(parent_idx, dtype=np.int32)
+        tok = np.zeros(len(par), dtype=np.int32)
+        pr = np.zeros(len(par), dtype=np.float32)
+        rc = lib().ssd_trigram_propose(self.h, int(prev1), int(root), par.ctypes.data, len(par), tok.ctypes.data, pr.ctypes.data)
+        if rc != SSD_OK:
+            raise SsdError(rc)
+        return tok, pr
+
+    def contexts(self) -> int:
+        c = C.c_int64(0)
+        rc = lib().ssd_trigram_contexts(self.h, C.byref(c))
+        if rc != SSD_OK:
+            raise SsdError(rc)
+        return c.value
+
+    def close(self):
+        if self.h:
+            lib().ssd_trigram_destroy(self.h)
+            self.h = None
