@@ -185,6 +185,32 @@ int ssd_accept_tree_noalloc(int device, void *cuda_stream, const float *logits, 
                             int32_t *path_out, int32_t *n_path_out, int32_t *next_token_out);
 
 /*
+ * ssd_accept_tree with the proposal rows given as short index / value lists instead of dense rows: row c is zero except
+ * row c[row_idx[c][e]] = row_val[c][e], e < entries (host arrays [n_nodes][entries], entries <= 1024; an index < 0 marks an
+ * unused slot).  A deterministic proposal ("the second or third most likely tokens", Section 3.1) is a one-entry row with
+ * value 1, a trigram row has four entries.  The rows are expanded on the device and the walk of ssd_accept_tree runs on
+ * them: same rule, same results, same errors.
+ */
+int ssd_accept_tree_sparse(ssd_ctx *ctx, const float *logits, const int32_t *row_idx, const float *row_val, int32_t entries,
+                           const int32_t *tokens, const int32_t *parent_idx, int32_t n_nodes, const ssd_sampling *sampling, ssd_rng *rng_state,
+                           int32_t *path_out, int32_t *n_path_out, int32_t *next_token_out);
+
+/*
+ * What a stage proposes to the stage above it (Section 3.1: a tree of likely continuations is built from the lower
+ * model's distributions; Section 3.2: the lower model may itself be the verifier of a still lower one).  For each of the
+ * `m` listed nodes of a verified tree (nodes: host [m], logits: DEVICE [*, vocab] as written by ssd_verify_tree):
+ *   - the node's next-token law, exactly the target law ssd_accept_tree gives that node (fp64 softmax of logits /
+ *     temperature over the entries kept by the top-k cut), written as an fp32 row to rows_out[j] (DEVICE [m, vocab];
+ *     may be NULL) - the proposal row of children proposed from it;
+ *   - `picks` (0..8) candidate next tokens, tokens_out (host [m][picks]): mode SSD_GREEDY, the most probable tokens in
+ *     order (ties towards the lower id); mode SSD_SAMPLING, independent inverse-CDF draws from the law with the uniforms
+ *     u(seed, step, 1024 + 16 node + t) of rng_state (Philox4x32-10 as in ssd_accept_tree).
+ * Increments rng_state->step.  Waits for the stream.  Errors: BAD_ARG (also: a listed row holds a non-finite logit), NOMEM, CUDA.
+ */
+int ssd_propose_children(ssd_ctx *ctx, const float *logits, const int32_t *nodes, int32_t m, int32_t picks, const ssd_sampling *sampling,
+                         ssd_rng *rng_state, float *rows_out, int32_t *tokens_out);
+
+/*
  * Append the accepted slices (Section 3.1): for every layer, scratch row kv_len + path[j] becomes
  * committed row kv_len + j, in place; kv_len += n_path.  `path` (host) must start at the root and
  * each entry must be a child of the one before in the tree of the last ssd_verify_tree on `kv`

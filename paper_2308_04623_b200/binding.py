@@ -18,7 +18,7 @@ SSD_TUNE_CLUSTER_QKV, SSD_TUNE_CLUSTER_O, SSD_TUNE_CLUSTER_FC, SSD_TUNE_CLUSTER_
 
 # every symbol include/ssd.h declares
 EXPORTS = ("ssd_create", "ssd_load_weights", "ssd_kv_create", "ssd_kv_reset", "ssd_kv_len", "ssd_kv_rollback",
-           "ssd_kv_destroy", "ssd_verify_tree", "ssd_accept_tree", "ssd_kv_commit", "ssd_kv_read", "ssd_strerror",
+           "ssd_kv_destroy", "ssd_verify_tree", "ssd_accept_tree", "ssd_accept_tree_sparse", "ssd_propose_children", "ssd_kv_commit", "ssd_kv_read", "ssd_strerror",
            "ssd_last_device_status", "ssd_reset_device_status", "ssd_debug_expire_wait", "ssd_last_cuda_error", "ssd_last_cuda_error_line", "ssd_kernel_launches", "ssd_set_tuning", "ssd_get_phase_trace", "ssd_accept_tree_noalloc", "ssd_destroy",
            "ssd_trigram_build", "ssd_trigram_lookup", "ssd_trigram_propose", "ssd_trigram_contexts", "ssd_trigram_destroy")
 
@@ -74,6 +74,9 @@ def lib():
         L.ssd_accept_tree_noalloc.argtypes = [C.c_int, _VP, _VP, _VP, _VP, _VP, C.c_int32, C.c_int32, C.POINTER(ssd_sampling),
                                               C.POINTER(ssd_rng), _VP, C.POINTER(C.c_int32), C.POINTER(C.c_int32)]
         L.ssd_kv_commit.argtypes = [_VP, _VP, _VP, C.c_int32]
+        L.ssd_accept_tree_sparse.argtypes = [_VP, _VP, _VP, _VP, C.c_int32, _VP, _VP, C.c_int32, C.POINTER(ssd_sampling), C.POINTER(ssd_rng),
+                                             _VP, C.POINTER(C.c_int32), C.POINTER(C.c_int32)]
+        L.ssd_propose_children.argtypes = [_VP, _VP, _VP, C.c_int32, C.c_int32, C.POINTER(ssd_sampling), C.POINTER(ssd_rng), _VP, _VP]
         L.ssd_kv_read.argtypes = [_VP, _VP, C.c_int32, C.c_int32, C.c_int32, C.c_int32, _VP]
         L.ssd_strerror.argtypes = [C.c_int]
         L.ssd_strerror.restype = C.c_char_p
@@ -175,6 +178,34 @@ class Context:
                                    C.byref(samp), C.byref(rng), path.ctypes.data, C.byref(n_path), C.byref(nxt))
         self._chk(rc)
         return [int(v) for v in path[:n_path.value]], int(nxt.value)
+
+    def accept_tree_sparse(self, logits_ptr: int, row_idx, row_val, tokens, parent_idx, mode: int = SSD_SAMPLING, temperature: float = 1.0,
+                           top_k: int = 0, rng: ssd_rng | None = None):
+        """ssd_accept_tree_sparse: proposal rows as [n, entries] index / value lists (index < 0 = unused slot)."""
+        tokens, parent_idx = _i32(tokens), _i32(parent_idx)
+        n = len(tokens)
+        idx = np.ascontiguousarray(row_idx, dtype=np.int32).reshape(n, -1)
+        val = np.ascontiguousarray(row_val, dtype=np.float32).reshape(n, -1)
+        assert idx.shape == val.shape
+        samp = ssd_sampling(mode, temperature, top_k)
+        rng = rng if rng is not None else ssd_rng(0, 0)
+        path = np.zeros(max(n, 1), dtype=np.int32)
+        n_path, nxt = C.c_int32(0), C.c_int32(-1)
+        rc = lib().ssd_accept_tree_sparse(self.h, _VP(logits_ptr), idx.ctypes.data, val.ctypes.data, idx.shape[1], tokens.ctypes.data,
+                                          parent_idx.ctypes.data, n, C.byref(samp), C.byref(rng), path.ctypes.data, C.byref(n_path), C.byref(nxt))
+        self._chk(rc)
+        return [int(v) for v in path[:n_path.value]], int(nxt.value)
+
+    def propose_children(self, logits_ptr: int, nodes, picks: int, mode: int = SSD_GREEDY, temperature: float = 1.0, top_k: int = 0,
+                         rng: ssd_rng | None = None, rows_out_ptr: int = 0) -> np.ndarray:
+        """ssd_propose_children.  Returns tokens int32 [len(nodes), picks]; the nodes' laws go to ``rows_out_ptr`` (device) if given."""
+        nodes = _i32(nodes)
+        samp = ssd_sampling(mode, temperature, top_k)
+        rng = rng if rng is not None else ssd_rng(0, 0)
+        out = np.zeros((len(nodes), max(picks, 1)), dtype=np.int32)
+        self._chk(lib().ssd_propose_children(self.h, _VP(logits_ptr), nodes.ctypes.data, len(nodes), picks, C.byref(samp), C.byref(rng),
+                                             _VP(rows_out_ptr or 0), out.ctypes.data))
+        return out[:, :picks]
 
     def kv_commit(self, kv: "KV", path):
         path = _i32(path)

@@ -252,6 +252,48 @@ __global__ void __launch_bounds__(ACC_THREADS) row_law_kernel(const float *__res
     }
 }
 
+// Inverse-CDF draw from r (fp64, not necessarily normalised) by the whole CTA: ONE thread writes to *token_out the smallest v
+// whose running sum exceeds u * sum(r); if rounding leaves none, the largest v with r[v] > 0.
+__device__ void draw_from(const double *__restrict__ r, int V, double u, int32_t *__restrict__ token_out, BlockScratch &s) {
+    const int tid = threadIdx.x;
+    const int chunk = (V + ACC_THREADS - 1) / ACC_THREADS;
+    const int v0 = min(V, tid * chunk), v1 = min(V, v0 + chunk);
+    double csum = 0.0;
+    int last_pos = -1;
+    for (int v = v0; v < v1; ++v) { csum += r[v]; if (r[v] > 0.0) last_pos = v; }
+    // inclusive scan of the chunk sums over the block
+    double incl = csum;
+#pragma unroll
+    for (int off = 1; off < 32; off <<= 1) {
+        const double t = __shfl_up_sync(0xffffffffu, incl, off);
+        if ((tid & 31) >= off) incl += t;
+    }
+    __syncthreads();
+    if ((tid & 31) == 31) s.d[tid >> 5] = incl;
+    __syncthreads();
+    double warp_base = 0.0, total = 0.0;
+    for (int w = 0; w < ACC_THREADS / 32; ++w) {
+        if (w < (tid >> 5)) warp_base += s.d[w];
+        total += s.d[w];
+    }
+    incl += warp_base;
+    const double target = u * total;
+    const int first = block_min_int(incl > target ? tid : 0x7fffffff, s);
+    const int fallback = block_max_int(last_pos, s);
+    if (first == 0x7fffffff) {
+        if (tid == 0) *token_out = fallback;
+    } else if (tid == first) {
+        double run = incl - csum;
+        int pick = -1, lp = -1;
+        for (int v = v0; v < v1; ++v) {
+            if (r[v] > 0.0) lp = v;
+            run += r[v];
+            if (run > target) { pick = v; break; }
+        }
+        *token_out = pick >= 0 ? pick : lp;
+    }
+}
+
 // What happens at node `cur`, whose target law is r (with its support list sup[0..cnt) if cnt >= 0): its children are
 // tried in index order, each refusal replacing r by the renormalised residual.  Returns the accepted child (the same
 // value in every thread), or -1 after ONE thread has written the extra token, drawn from r by inverse CDF, to *token_out.
@@ -305,42 +347,7 @@ __device__ int node_decide(double *__restrict__ r, int cnt, const int32_t *__res
         }
         return -1;
     }
-    const int chunk = (V + ACC_THREADS - 1) / ACC_THREADS;
-    const int v0 = min(V, tid * chunk), v1 = min(V, v0 + chunk);
-    double csum = 0.0;
-    int last_pos = -1;
-    for (int v = v0; v < v1; ++v) { csum += r[v]; if (r[v] > 0.0) last_pos = v; }
-    // inclusive scan of the chunk sums over the block
-    double incl = csum;
-#pragma unroll
-    for (int off = 1; off < 32; off <<= 1) {
-        const double t = __shfl_up_sync(0xffffffffu, incl, off);
-        if ((tid & 31) >= off) incl += t;
-    }
-    __syncthreads();
-    if ((tid & 31) == 31) s.d[tid >> 5] = incl;
-    __syncthreads();
-    double warp_base = 0.0, total = 0.0;
-    for (int w = 0; w < ACC_THREADS / 32; ++w) {
-        if (w < (tid >> 5)) warp_base += s.d[w];
-        total += s.d[w];
-    }
-    incl += warp_base;
-    const double target = u * total;
-    const int first = block_min_int(incl > target ? tid : 0x7fffffff, s);
-    const int fallback = block_max_int(last_pos, s);
-    if (first == 0x7fffffff) {
-        if (tid == 0) *token_out = fallback;
-    } else if (tid == first) {
-        double run = incl - csum;
-        int pick = -1, lp = -1;
-        for (int v = v0; v < v1; ++v) {
-            if (r[v] > 0.0) lp = v;
-            run += r[v];
-            if (run > target) { pick = v; break; }
-        }
-        *token_out = pick >= 0 ? pick : lp;
-    }
+    draw_from(r, V, u, token_out, s);
     return -1;
 }
 
@@ -432,6 +439,80 @@ cudaError_t launch_accept(const float *logits, const float *draft_probs, const N
             *launches += 1;
         }
     }
+    return cudaGetLastError();
+}
+
+// ---------------------------------------------------------------------------------------------
+// Proposals of one stage for the stage above (Sections 3.1 / 3.2: a tree of likely continuations is assembled from
+// the lower model's distributions - "the second or third most likely tokens" - or from draws of them).  For each
+// listed node: its law (the same fp64 softmax with temperature and top-k cut that the acceptance rule uses as a
+// node's target), written out as an fp32 row if asked, and `picks` candidate next tokens: the most probable ones in
+// order (greedy), or independent inverse-CDF draws with the counter-based uniforms u(seed, step, 1024 + 16 node + t).
+// One CTA per listed node; `scratch` holds one fp64 row per CTA.
+// ---------------------------------------------------------------------------------------------
+__global__ void __launch_bounds__(ACC_THREADS) propose_children_kernel(const float *__restrict__ logits, NodeList nodes, int V, double temperature,
+                                                                       int top_k, int mode, int picks, uint64_t seed, uint64_t step,
+                                                                       double *__restrict__ scratch, float *__restrict__ rows_out,
+                                                                       int32_t *__restrict__ tokens_out, int32_t *__restrict__ bad_out) {
+    __shared__ BlockScratch s;
+    __shared__ int32_t s_pick;
+    const int j = blockIdx.x, node = nodes.v[j], tid = threadIdx.x;
+    double *r = scratch + (size_t)j * V;
+    const int bad = row_law(logits + (size_t)node * V, V, temperature, top_k, r, s);
+    if (tid == 0) bad_out[j] = bad;
+    if (bad) {
+        for (int t = tid; t < picks; t += ACC_THREADS) tokens_out[j * picks + t] = -1;
+        return;
+    }
+    if (rows_out)
+        for (int v = tid; v < V; v += ACC_THREADS) rows_out[(size_t)j * V + v] = (float)r[v];
+    for (int t = 0; t < picks; ++t) {
+        if (mode == SSD_GREEDY) { // the most probable token not yet picked; ties towards the lower id
+            double best = -1.0;
+            int arg = 0x7fffffff;
+            for (int v = tid; v < V; v += ACC_THREADS)
+                if (r[v] > best) { best = r[v]; arg = v; } // (ascending v per thread: the first maximum is the lowest id)
+            const double top = block_max(best, s);
+            const int pick = block_min_int(best == top ? arg : 0x7fffffff, s);
+            if (tid == 0) { tokens_out[j * picks + t] = pick; r[pick] = -1.0; }
+            __syncthreads();
+        } else {
+            const double u = uniform24(seed, step, 1024u + 16u * (uint32_t)node + (uint32_t)t);
+            draw_from(r, V, u, &s_pick, s);
+            __syncthreads();
+            if (tid == 0) tokens_out[j * picks + t] = s_pick;
+        }
+    }
+}
+
+cudaError_t launch_propose_children(const float *logits, const NodeList &nodes, int m, int vocab, int mode, float temperature, int top_k, int picks,
+                                    uint64_t seed, uint64_t step, double *scratch, float *rows_out, int32_t *tokens_out, int32_t *bad_out,
+                                    cudaStream_t s) {
+    propose_children_kernel<<<m, ACC_THREADS, 0, s>>>(logits, nodes, vocab, (double)temperature, top_k, mode, picks, seed, step, scratch, rows_out,
+                                                      tokens_out, bad_out);
+    return cudaGetLastError();
+}
+
+// rows[j, :] = 0 except rows[j, idx[j, e]] = val[j, e] for the listed entries (idx < 0: unused slot): proposal rows given
+// as short index / value lists (a trigram row has four non-zeros, a deterministic proposal one) made dense for the
+// acceptance kernels.  One CTA per row.
+__global__ void __launch_bounds__(256) expand_sparse_rows_kernel(const int32_t *__restrict__ idx, const float *__restrict__ val, int entries, int V,
+                                                                 float *__restrict__ rows) {
+    float *row = rows + (size_t)blockIdx.x * V;
+    if ((V & 3) == 0 && (reinterpret_cast<uintptr_t>(row) & 15) == 0) {
+        float4 *r4 = reinterpret_cast<float4 *>(row);
+        for (int v = threadIdx.x; v < V / 4; v += 256) r4[v] = make_float4(0.f, 0.f, 0.f, 0.f);
+    } else {
+        for (int v = threadIdx.x; v < V; v += 256) row[v] = 0.f;
+    }
+    __syncthreads();
+    for (int e = threadIdx.x; e < entries; e += 256) {
+        const int v = idx[(size_t)blockIdx.x * entries + e];
+        if (v >= 0 && v < V) row[v] = val[(size_t)blockIdx.x * entries + e];
+    }
+}
+cudaError_t launch_expand_sparse_rows(const int32_t *idx, const float *val, int n, int entries, int vocab, float *rows, cudaStream_t s) {
+    expand_sparse_rows_kernel<<<n, 256, 0, s>>>(idx, val, entries, vocab, rows);
     return cudaGetLastError();
 }
 

@@ -59,6 +59,11 @@ struct ssd_ctx {
     cudaStream_t capture_stream;
     AcceptScratch acc;
     int32_t *h_result; // pinned host copy of acc.result
+    int32_t *h_propose; // pinned: picks of ssd_propose_children [SSD_MAX_NODES * 8] then one non-finite flag per listed node
+    // proposal rows given as index / value lists: device copies of the lists and the dense rows they expand to (grown on demand)
+    int32_t *d_sparse_idx;
+    float *d_sparse_val, *d_sparse_rows;
+    size_t sparse_entries_cap, sparse_rows_cap;
     int32_t *d_status;
 };
 
@@ -315,6 +320,25 @@ int capture_forward(ssd_ctx *ctx, int n, int cap, const NodeList &tk, const Node
     fg.kernels = kernels;
     return SSD_OK;
 }
+// Per-row fp64 scratch of the sampling rule and of the proposal laws, [rows, vocab], with the support lists of the top-k
+// cut behind it; grown on first use and when a larger tree arrives (a failed allocation only means that the acceptance
+// walk computes the visited rows itself).
+int ensure_law_rows(ssd_ctx *ctx, int n) {
+    if (ctx->acc.rows_cap >= n) return SSD_OK;
+    CU(cudaStreamSynchronize(ctx->stream));
+    if (ctx->acc.rows) { cudaFree(ctx->acc.rows); ctx->acc.rows = nullptr; ctx->acc.rows_cap = 0; ctx->acc.sup_idx = ctx->acc.sup_cnt = nullptr; }
+    const int rows = (n + 31) & ~31;
+    const size_t law_bytes = (size_t)rows * ctx->cfg.vocab * sizeof(double), idx_bytes = (size_t)rows * SSD_ACC_SUPPORT * sizeof(int32_t);
+    void *q = nullptr;
+    if (cudaMalloc(&q, law_bytes + idx_bytes + (size_t)rows * sizeof(int32_t)) == cudaSuccess) {
+        ctx->acc.rows = (double *)q; ctx->acc.rows_cap = rows;
+        ctx->acc.sup_idx = (int32_t *)((char *)q + law_bytes);
+        ctx->acc.sup_cnt = (int32_t *)((char *)q + law_bytes + idx_bytes);
+    } else {
+        (void)cudaGetLastError();
+    }
+    return SSD_OK;
+}
 } // namespace
 
 extern "C" {
@@ -357,6 +381,9 @@ int ssd_create(const ssd_config *cfg, int device, void *cuda_stream, ssd_ctx **o
     ctx->launches = 0;
     ctx->elt = cfg->dtype == SSD_DTYPE_F32 ? 4 : 2;
     ctx->h_result = nullptr;
+    ctx->h_propose = nullptr;
+    ctx->d_sparse_idx = nullptr; ctx->d_sparse_val = nullptr; ctx->d_sparse_rows = nullptr;
+    ctx->sparse_entries_cap = ctx->sparse_rows_cap = 0;
     DeviceGuard g(device);
     int rc = g.ok ? SSD_OK : SSD_ERR_CUDA;
     const size_t n = cfg->max_nodes, d = cfg->d_model;
@@ -416,6 +443,7 @@ int ssd_create(const ssd_config *cfg, int device, void *cuda_stream, ssd_ctx **o
     }
     if (rc == SSD_OK) {
         cudaError_t e = cudaMallocHost((void **)&ctx->h_result, sizeof(int32_t) * (n + 4));
+        if (e == cudaSuccess) e = cudaMallocHost((void **)&ctx->h_propose, sizeof(int32_t) * SSD_MAX_NODES * 9);
         if (e == cudaSuccess) e = cudaMemsetAsync(ctx->d_status, 0, sizeof(int32_t), ctx->stream);
         if (e != cudaSuccess) rc = fail_cuda(ctx, e);
     }
@@ -434,6 +462,8 @@ void ssd_destroy(ssd_ctx *ctx) {
     for (void *p : ctx->owned) cudaFree(p);
     if (ctx->acc.rows) cudaFree(ctx->acc.rows);
     if (ctx->h_result) cudaFreeHost(ctx->h_result);
+    if (ctx->h_propose) cudaFreeHost(ctx->h_propose);
+    cudaFree(ctx->d_sparse_idx); cudaFree(ctx->d_sparse_val); cudaFree(ctx->d_sparse_rows);
     delete ctx;
 }
 
@@ -620,21 +650,9 @@ int ssd_accept_tree(ssd_ctx *ctx, const float *logits, const float *draft_probs,
     NodeList tk, pr;
     memcpy(tk.v, tokens, sizeof(int32_t) * n);
     memcpy(pr.v, parent_idx, sizeof(int32_t) * n);
-    if (sampling->mode == SSD_SAMPLING && n > 1 && ctx->acc.rows_cap < n) {
-        // Per-row scratch of the sampling rule, [rows, vocab] fp64, grown on first use and when a larger tree arrives (a
-        // failed allocation only means that the walk computes the visited rows itself).
-        CU(cudaStreamSynchronize(ctx->stream));
-        if (ctx->acc.rows) { cudaFree(ctx->acc.rows); ctx->acc.rows = nullptr; ctx->acc.rows_cap = 0; ctx->acc.sup_idx = ctx->acc.sup_cnt = nullptr; }
-        const int rows = (n + 31) & ~31;
-        const size_t law_bytes = (size_t)rows * c.vocab * sizeof(double), idx_bytes = (size_t)rows * SSD_ACC_SUPPORT * sizeof(int32_t);
-        void *q = nullptr;
-        if (cudaMalloc(&q, law_bytes + idx_bytes + (size_t)rows * sizeof(int32_t)) == cudaSuccess) {
-            ctx->acc.rows = (double *)q; ctx->acc.rows_cap = rows;
-            ctx->acc.sup_idx = (int32_t *)((char *)q + law_bytes);
-            ctx->acc.sup_cnt = (int32_t *)((char *)q + law_bytes + idx_bytes);
-        } else {
-            (void)cudaGetLastError();
-        }
+    if (sampling->mode == SSD_SAMPLING && n > 1) {
+        rc = ensure_law_rows(ctx, n);
+        if (rc != SSD_OK) return rc;
     }
     int launched = 0;
     AcceptScratch sc = ctx->acc;
@@ -655,6 +673,62 @@ int ssd_accept_tree(ssd_ctx *ctx, const float *logits, const float *draft_probs,
     // ssd_reset_device_status): the logits this walk read are not to be trusted.
     if (ctx->h_result[3] != 0) return SSD_ERR_TIMEOUT;
     return ctx->h_result[2];
+}
+
+int ssd_accept_tree_sparse(ssd_ctx *ctx, const float *logits, const int32_t *row_idx, const float *row_val, int32_t entries,
+                           const int32_t *tokens, const int32_t *parent_idx, int32_t n_nodes, const ssd_sampling *sampling, ssd_rng *rng_state,
+                           int32_t *path_out, int32_t *n_path_out, int32_t *next_token_out) {
+    if (!ctx || !row_idx || !row_val || entries < 1 || entries > SSD_ACC_SUPPORT || n_nodes < 1 || n_nodes > SSD_MAX_NODES) return SSD_ERR_BAD_ARG;
+    DeviceGuard g(ctx->device);
+    if (!g.ok) return SSD_ERR_CUDA;
+    const size_t need_e = (size_t)n_nodes * entries, need_r = (size_t)n_nodes * ctx->cfg.vocab;
+    if (ctx->sparse_entries_cap < need_e) {
+        CU(cudaStreamSynchronize(ctx->stream));
+        cudaFree(ctx->d_sparse_idx); cudaFree(ctx->d_sparse_val);
+        ctx->d_sparse_idx = nullptr; ctx->d_sparse_val = nullptr; ctx->sparse_entries_cap = 0;
+        CU(cudaMalloc((void **)&ctx->d_sparse_idx, need_e * sizeof(int32_t)));
+        CU(cudaMalloc((void **)&ctx->d_sparse_val, need_e * sizeof(float)));
+        ctx->sparse_entries_cap = need_e;
+    }
+    if (ctx->sparse_rows_cap < need_r) {
+        CU(cudaStreamSynchronize(ctx->stream));
+        cudaFree(ctx->d_sparse_rows);
+        ctx->d_sparse_rows = nullptr; ctx->sparse_rows_cap = 0;
+        CU(cudaMalloc((void **)&ctx->d_sparse_rows, need_r * sizeof(float)));
+        ctx->sparse_rows_cap = need_r;
+    }
+    CU(cudaMemcpyAsync(ctx->d_sparse_idx, row_idx, need_e * sizeof(int32_t), cudaMemcpyHostToDevice, ctx->stream));
+    CU(cudaMemcpyAsync(ctx->d_sparse_val, row_val, need_e * sizeof(float), cudaMemcpyHostToDevice, ctx->stream));
+    CU(launch_expand_sparse_rows(ctx->d_sparse_idx, ctx->d_sparse_val, n_nodes, entries, ctx->cfg.vocab, ctx->d_sparse_rows, ctx->stream));
+    ctx->launches += 1;
+    // (the lists are pageable host memory: the copies above have read them by the time the calls return)
+    return ssd_accept_tree(ctx, logits, ctx->d_sparse_rows, tokens, parent_idx, n_nodes, sampling, rng_state, path_out, n_path_out, next_token_out);
+}
+
+int ssd_propose_children(ssd_ctx *ctx, const float *logits, const int32_t *nodes, int32_t m, int32_t picks, const ssd_sampling *sampling,
+                         ssd_rng *rng_state, float *rows_out, int32_t *tokens_out) {
+    if (!ctx || !logits || !nodes || !sampling || !rng_state || !tokens_out || m < 1 || m > SSD_MAX_NODES || picks < 0 || picks > 8) return SSD_ERR_BAD_ARG;
+    if (sampling->mode != SSD_GREEDY && sampling->mode != SSD_SAMPLING) return SSD_ERR_BAD_ARG;
+    if (!(sampling->temperature > 0.f) || sampling->top_k < 0) return SSD_ERR_BAD_ARG;
+    for (int j = 0; j < m; ++j)
+        if (nodes[j] < 0 || nodes[j] >= SSD_MAX_NODES) return SSD_ERR_BAD_ARG;
+    DeviceGuard g(ctx->device);
+    if (!g.ok) return SSD_ERR_CUDA;
+    int rc = ensure_law_rows(ctx, m);
+    if (rc != SSD_OK) return rc;
+    if (ctx->acc.rows_cap < m) return SSD_ERR_NOMEM;
+    NodeList nl;
+    memcpy(nl.v, nodes, sizeof(int32_t) * m);
+    int32_t *picks_host = ctx->h_propose, *bad_host = ctx->h_propose + SSD_MAX_NODES * 8; // the kernel writes into pinned host memory
+    CU(launch_propose_children(logits, nl, m, ctx->cfg.vocab, sampling->mode, sampling->temperature, sampling->top_k, picks, rng_state->seed,
+                               rng_state->step, ctx->acc.rows, rows_out, picks_host, bad_host, ctx->stream));
+    ctx->launches += 1;
+    CU(cudaStreamSynchronize(ctx->stream));
+    rng_state->step += 1;
+    for (int j = 0; j < m; ++j)
+        if (bad_host[j]) return SSD_ERR_BAD_ARG; // a listed row holds a non-finite logit
+    memcpy(tokens_out, picks_host, sizeof(int32_t) * m * picks);
+    return SSD_OK;
 }
 
 int ssd_kv_commit(ssd_ctx *ctx, ssd_kv *kv, const int32_t *path, int32_t n_path) {

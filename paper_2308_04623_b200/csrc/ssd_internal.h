@@ -142,6 +142,10 @@ struct AcceptScratch {
     int32_t *result;    // [max_nodes + 4]: n_path, next_token, status, device error word, path[...]
     const int32_t *dev_status; // the forward's device error word (copied into result[3] by the walk) or null
 };
+cudaError_t launch_propose_children(const float *logits, const NodeList &nodes, int m, int vocab, int mode, float temperature, int top_k, int picks,
+                                    uint64_t seed, uint64_t step, double *scratch, float *rows_out, int32_t *tokens_out, int32_t *bad_out,
+                                    cudaStream_t s);
+cudaError_t launch_expand_sparse_rows(const int32_t *idx, const float *val, int n, int entries, int vocab, float *rows, cudaStream_t s);
 cudaError_t launch_expired_wait(int32_t *status, long long limit_cycles, cudaStream_t s);
 cudaError_t launch_accept(const float *logits, const float *draft_probs, const NodeList &tokens, const NodeList &parent, int n,
                           int vocab, int mode, float temperature, int top_k, uint64_t seed, uint64_t step,

@@ -608,3 +608,75 @@ def test_expired_device_wait_surfaces_as_timeout_and_can_be_reset(util, ssd):
         assert (path, nxt) == (opath, onxt)
     finally:
         p.close()
+
+
+# --------------------------------------------------------------------------- proposal rows as lists, proposals of a stage
+def test_sparse_proposal_rows_give_the_dense_rule_on_the_trigram_tree(ssd):
+    """ssd_accept_tree_sparse on the stage-two tree: the four-entry trigram rows and one-entry (deterministic) rows walk exactly
+    as the oracle's dense rule does on the same rows written out densely, at the full vocabulary."""
+    cfg = ssd_synth.config("gpt2_small")
+    V = cfg["vocab"]
+    ctx = ssd.Context(cfg, device=0, stream=torch.cuda.current_stream().cuda_stream)
+    try:
+        rng = np.random.default_rng(33)
+        tokens, parent, dense = ssd_synth.trigram_tree(11, 22, 33, V)
+        n = len(parent)
+        logits = rng.normal(0.0, 1.5, size=(n, V)).astype(np.float32)
+        for c in range(1, n):                       # make the proposed tokens plausible under the verifier
+            logits[parent[c], tokens[c]] += 6.0
+        idx = np.full((n, 4), -1, dtype=np.int32)
+        val = np.zeros((n, 4), dtype=np.float32)
+        for c in range(1, n):
+            nz = np.nonzero(dense[c])[0]
+            idx[c, :len(nz)], val[c, :len(nz)] = nz, dense[c, nz]
+        onehot = np.zeros((n, V), dtype=np.float32)
+        onehot[np.arange(1, n), tokens[1:]] = 1.0
+        lg = torch.from_numpy(logits).cuda()
+        deep = 0
+        for step in range(40):
+            for rows_dense, i_, v_ in ((dense, idx, val), (onehot, np.concatenate([[-1], tokens[1:]]).reshape(-1, 1), np.ones((n, 1), dtype=np.float32))):
+                for top_k in (0, 50):
+                    got = ctx.accept_tree_sparse(lg.data_ptr(), i_, v_, tokens, parent, mode=ssd.SSD_SAMPLING, top_k=top_k, rng=ssd.binding.ssd_rng(3, step))
+                    opath, onxt, margin = ssd_oracle.accept_tree(logits, rows_dense, tokens, parent, mode=1, top_k=top_k, seed=3, step=step)
+                    assert got == (opath, onxt), (step, top_k, margin)
+                    deep += len(opath) > 1
+        assert deep > 20
+    finally:
+        ctx.close()
+
+
+def test_proposed_children_follow_the_nodes_laws(ssd):
+    """ssd_propose_children: the rows are the nodes' target laws (fp64 softmax, temperature, top-k cut) to fp32 rounding, the
+    deterministic picks are the most probable tokens in order, the sampled picks are the inverse-CDF draws of the same uniforms."""
+    from oracle import staged_oracle
+    cfg = ssd_synth.config("tiny", vocab=5000)
+    V = cfg["vocab"]
+    ctx = ssd.Context(cfg, device=0, stream=torch.cuda.current_stream().cuda_stream)
+    try:
+        rng = np.random.default_rng(8)
+        logits = rng.normal(0.0, 2.0, size=(12, V)).astype(np.float32)
+        logits[3, [7, 9]] = 11.0                         # a tie at the top: the lower id comes first
+        lg = torch.from_numpy(logits).cuda()
+        nodes = [0, 3, 11, 5]
+        rows = torch.zeros((len(nodes), V), dtype=torch.float32, device="cuda")
+        for T, k in ((1.0, 0), (0.7, 50)):
+            srng = ssd.binding.ssd_rng(21, 4)
+            got = ctx.propose_children(lg.data_ptr(), nodes, 4, mode=ssd.SSD_GREEDY, temperature=T, top_k=k, rng=srng, rows_out_ptr=rows.data_ptr())
+            assert srng.step == 5
+            r = rows.cpu().numpy()
+            for j, node in enumerate(nodes):
+                p = staged_oracle.law(logits[node], float(np.float32(T)), k)
+                assert np.abs(r[j].astype(np.float64) - p).max() <= 1e-7 * max(1.0, p.max())
+                assert got[j].tolist() == staged_oracle.most_probable(p, 4)
+            assert got[1, :2].tolist() == [7, 9]
+            got = ctx.propose_children(lg.data_ptr(), nodes, 8, mode=ssd.SSD_SAMPLING, temperature=T, top_k=k, rng=ssd.binding.ssd_rng(21, 9))
+            for j, node in enumerate(nodes):
+                p = staged_oracle.law(logits[node], float(np.float32(T)), k)
+                assert got[j].tolist() == [staged_oracle.draw(p, ssd_oracle.uniform(21, 9, 1024 + 16 * node + t)) for t in range(8)]
+        bad = lg.clone()
+        bad[5, 100] = float("inf")
+        with pytest.raises(ssd.SsdError) as e:
+            ctx.propose_children(bad.data_ptr(), nodes, 2)
+        assert e.value.code == ssd.SSD_ERR_BAD_ARG
+    finally:
+        ctx.close()
