@@ -74,7 +74,7 @@ class StagedOracle:
         self.rng_step = 0
         self.seq = []
         self.min_margin = float("inf")
-        self.stats = {"oracle_steps": 0, "draft_forwards": 0, "emitted": 0, "origin": {"trigram": 0, "draft": 0, "oracle": 0}}
+        self.stats = {"target_steps": 0, "draft_forwards": 0, "emitted": 0, "origin": {"trigram": 0, "draft": 0, "target": 0}}
 
     def next_step(self) -> int:
         s = self.rng_step
@@ -147,11 +147,11 @@ class StagedOracle:
         self.min_margin = min(self.min_margin, margin)
         self.kv0.commit(path0)
         emitted = [int(tokens1[c]) for c in path0[1:]] + [int(next0)]
-        origins = [origin1[c] for c in path0[1:]] + ["oracle"]
+        origins = [origin1[c] for c in path0[1:]] + ["target"]
         k = sum(1 for j, c in enumerate(path0[1:], start=1) if c == j)     # chain tokens the oracle accepted
         self.kv1.rollback(len(seq_old) + min(k, m - 1))
         self.seq = seq_old + emitted
-        self.stats["oracle_steps"] += 1
+        self.stats["target_steps"] += 1
         self.stats["emitted"] += len(emitted)
         for o in origins:
             self.stats["origin"][o] += 1

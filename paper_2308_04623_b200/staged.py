@@ -1,6 +1,6 @@
 """The full staged decoding loop on the device (Section 3 of the paper), sequenced through the C ABI.
 
-Three stages: the oracle model, a small draft model and a trigram table (Section 4).  This module holds
+Three stages: the large model whose output the method preserves (the paper's top-level model, called the target here), a small draft model and a trigram table (Section 4).  This module holds
 no arithmetic: every forward, every acceptance decision, every proposal law, every draw and every table
 look-up is a kernel of libssd reached through `binding`; what is left here is the bookkeeping of which node
 hangs under which (lists of small integers) and the order of the calls.  torch is used for device buffers
@@ -13,7 +13,7 @@ One step:
       ssd_propose_children returns the draft's law at every node of the accepted path - the proposal rows of
       the chain for the next stage - and the sibling leaves of each level; ssd_kv_commit appends the accepted
       slices to the draft's cache speculatively.
-  stage 1 -> 0 (Section 3.1): the oracle scores the chain plus its sibling leaves in one ssd_verify_tree,
+  stage 1 -> 0 (Section 3.1): the target model scores the chain plus its sibling leaves in one ssd_verify_tree,
       ssd_accept_tree walks it, ssd_kv_commit appends the accepted slices, and ssd_kv_rollback takes the
       draft's cache back to what both models accepted.
 """
@@ -27,14 +27,14 @@ TRI_PARENT = np.array([-1, 0, 0, 0, 1, 1, 4, 6], dtype=np.int32)
 
 
 class StagedDecoder:
-    def __init__(self, oracle_ctx: B.Context, draft_ctx: B.Context, trigram: B.Trigram, mode: int = B.SSD_GREEDY, temperature: float = 1.0,
+    def __init__(self, target_ctx: B.Context, draft_ctx: B.Context, trigram: B.Trigram, mode: int = B.SSD_GREEDY, temperature: float = 1.0,
                  top_k: int = 0, rounds: int = 2, siblings: int = 1, seed: int = 0):
         import torch
         self.torch = torch
-        self.c0, self.c1, self.tri = oracle_ctx, draft_ctx, trigram
-        self.kv0, self.kv1 = oracle_ctx.new_kv(), draft_ctx.new_kv()
+        self.c0, self.c1, self.tri = target_ctx, draft_ctx, trigram
+        self.kv0, self.kv1 = target_ctx.new_kv(), draft_ctx.new_kv()
         self.mode, self.T, self.top_k, self.rounds, self.siblings = mode, float(np.float32(temperature)), top_k, rounds, siblings
-        self.V = oracle_ctx.cfg["vocab"]
+        self.V = target_ctx.cfg["vocab"]
         self.rng = B.ssd_rng(seed, 0)
         self.seq = []
         max_chain = rounds * len(TRI_PARENT)
@@ -42,7 +42,7 @@ class StagedDecoder:
         self.logits1 = torch.empty((len(TRI_PARENT) + 1, self.V), dtype=torch.float32, device="cuda")
         self.chain_rows = torch.zeros((max_chain + 1, self.V), dtype=torch.float32, device="cuda")   # row j: the law chain token j was proposed from
         self.rows1 = torch.zeros_like(self.logits0)
-        self.stats = {"oracle_steps": 0, "draft_forwards": 0, "emitted": 0, "origin": {"trigram": 0, "draft": 0, "oracle": 0}}
+        self.stats = {"target_steps": 0, "draft_forwards": 0, "emitted": 0, "origin": {"trigram": 0, "draft": 0, "target": 0}}
 
     def prefill(self, prompt):
         """Both caches take every prompt token but the last, which becomes the first root (hot-path calls only)."""
@@ -113,11 +113,11 @@ class StagedDecoder:
                                            top_k=self.top_k, rng=self.rng)
         self.c0.kv_commit(self.kv0, path0)
         emitted = [int(tokens1[c]) for c in path0[1:]] + [int(next0)]
-        origins = [origin1[c] for c in path0[1:]] + ["oracle"]
+        origins = [origin1[c] for c in path0[1:]] + ["target"]
         k = sum(1 for j, c in enumerate(path0[1:], start=1) if c == j)
         self.kv1.rollback(len(seq_old) + min(k, m - 1))
         self.seq = seq_old + emitted
-        self.stats["oracle_steps"] += 1
+        self.stats["target_steps"] += 1
         self.stats["emitted"] += len(emitted)
         for o in origins:
             self.stats["origin"][o] += 1

@@ -58,10 +58,10 @@ def test_greedy_staged_decoding_equals_greedy_autoregressive_decoding(draft_same
     want = staged_oracle.greedy_autoregressive(ssd_oracle.Model(cfg0, w0), PROMPT, n_tokens)
     assert got == want
     st = loop.stats
-    assert st["emitted"] >= n_tokens and st["draft_forwards"] == 2 * st["oracle_steps"]
-    assert sum(st["origin"].values()) == st["emitted"] and st["origin"]["oracle"] == st["oracle_steps"]
+    assert st["emitted"] >= n_tokens and st["draft_forwards"] == 2 * st["target_steps"]
+    assert sum(st["origin"].values()) == st["emitted"] and st["origin"]["target"] == st["target_steps"]
     if draft_same:   # the draft is the oracle: every chain token is accepted, several tokens per step
-        assert st["emitted"] / st["oracle_steps"] >= 3.0 and st["origin"]["trigram"] > 0 and st["origin"]["draft"] > 0
+        assert st["emitted"] / st["target_steps"] >= 3.0 and st["origin"]["trigram"] > 0 and st["origin"]["draft"] > 0
     assert len(loop.kv0) == len(loop.seq) - 1 and 1 <= len(loop.seq) - len(loop.kv1) <= 2
 
 
@@ -75,7 +75,7 @@ def test_sampled_staged_decoding_is_reproducible_and_keeps_both_caches_consisten
         loop.prefill(PROMPT)
         runs.append(loop.generate(60))
         assert all(0 <= t < cfg0["vocab"] for t in runs[-1])
-        assert loop.stats["emitted"] / loop.stats["oracle_steps"] > 1.2      # the oracle as its own draft: chains are accepted under sampling too
+        assert loop.stats["emitted"] / loop.stats["target_steps"] > 1.2      # the oracle as its own draft: chains are accepted under sampling too
         # the oracle's cache equals the cache of decoding the emitted sequence token by token
         ref = ssd_oracle.Model(cfg0, w0).new_kv()
         ref.prefill(np.asarray(loop.seq[:-1], dtype=np.int32), chunk=64)
