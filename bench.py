@@ -16,7 +16,8 @@ At one GPU the line also carries a `sweep` measured in the same process: the 16-
 trees on the same model, the stage-two verification of the GPT-2-small-shaped draft (512-token
 prefix, eight-node trigram tree) with a warm L2 and with an L2-evicting pass between steps, and the
 GPT-2-XL-shaped model over tree sizes 8..256 with the fractions of the HBM and tensor-core
-roofs and the tree size at which the tensor bound overtakes the HBM bound.
+roofs and the tree size at which the tensor bound overtakes the HBM bound, and the full staged loop
+(target, draft, trigram) at three controlled acceptance levels: tokens per target step and tokens/s.
 
 N > 1 runs N independent replicas (one process per GPU, no data-path collective): the path is a
 single sequence at batch 1 and does not shard.  Without torchrun's environment the script starts
@@ -415,6 +416,103 @@ def run_sweep(args, local, peaks):
     return out
 
 
+def run_staged(args, local, peaks, alphas=(0.3, 0.6, 0.9), n_tokens=256):
+    """The full staged loop at the benchmark's sizes with the acceptance made controllable: GPT-2-Large-shaped target,
+    GPT-2-small-shaped draft, a trigram table built from a synthetic stream.  Random-weight models never agree, so - as
+    the configuration defines it - every proposal row of the target's tree is alpha * softmax(target logits at the parent)
+    + (1 - alpha) * Dirichlet(0.5), children drawn independently from it; the harness obtains those rows by running the
+    target level by level (untimed).  What is timed, with CUDA events around each stage, is the method's own work per
+    step: the draft speculated by the trigram (rounds x [table look-up, draft verify of the eight-node tree, acceptance
+    with one-entry rows, the draft's laws and sibling picks, commit]), and the target's verify of the 32-node tree,
+    sampling acceptance and commit.  The draft's outputs do not feed the synthetic tree: this is the cost of the pipeline
+    at a controlled acceptance, not a language-model run."""
+    import torch
+    import paper_2308_04623_b200 as ssd
+    tgt = Runner(args.model, 64, local, args.tune, rng_seed=4004)
+    drf = Runner("gpt2_small", 64, local, args.tune, rng_seed=4004)
+    V = tgt.V
+    stream_tokens = np.random.default_rng(4).zipf(1.3, size=200000) % V
+    tri = ssd.Trigram(stream_tokens.astype(np.int32), V, device=local, stream=tgt.stream.cuda_stream)
+    parent = ssd_synth.tree_branching(32, tree_rule(32))
+    depth = ssd_synth.tree_depths(parent)
+    n = len(parent)
+    kids = {p: [c for c in range(n) if parent[c] == p] for p in range(n)}
+    tri_parent = ssd_synth.tree_chain_plus_branch()
+    rows = torch.zeros((n, V), dtype=torch.float32, device="cuda")
+    dlogits = torch.empty((16, V), dtype=torch.float32, device="cuda")
+    drows = torch.empty((16, V), dtype=torch.float32, device="cuda")
+    gen = torch.Generator(device="cuda")
+    out = {}
+    for alpha in alphas:
+        gen.manual_seed(int(alpha * 1000))
+        tgt.kv.rollback(64)
+        drf.kv.rollback(64)
+        srng = ssd.binding.ssd_rng(int(alpha * 100), 0)
+        seq = list(tgt.prefix) + [int(tgt.rng.integers(V))]
+        emitted, steps, t_draft, t_target, lengths = 0, 0, 0.0, 0.0, []
+        ev = [torch.cuda.Event(enable_timing=True) for _ in range(4)]
+        while emitted < n_tokens and len(tgt.kv) + 40 < tgt.cfg["n_ctx"]:
+            root = seq[-1]
+            # ---- timed: the draft stage (its results are not used for the synthetic tree)
+            base = len(drf.kv)
+            ev[0].record(tgt.stream)
+            for _ in range(2):
+                ttok, _ = tri.propose(seq[-2], root, tri_parent)
+                drf.ctx.verify_tree(ttok, tri_parent, drf.kv, dlogits.data_ptr())
+                idx = np.concatenate([[-1], ttok[1:]]).astype(np.int32).reshape(-1, 1)
+                path1, _ = drf.ctx.accept_tree_sparse(dlogits.data_ptr(), idx, np.ones((8, 1), dtype=np.float32), ttok, tri_parent,
+                                                       mode=ssd.SSD_SAMPLING, rng=srng)
+                drf.ctx.propose_children(dlogits.data_ptr(), path1, 1, mode=ssd.SSD_SAMPLING, rng=srng, rows_out_ptr=drows.data_ptr())
+                drf.ctx.kv_commit(drf.kv, path1)
+                drf.kv.rollback(base)
+            ev[1].record(tgt.stream)
+            # ---- untimed harness: the synthetic tree, level by level
+            tokens = np.zeros(n, dtype=np.int32)
+            tokens[0] = root
+            for d in range(int(depth.max())):
+                nd = int((depth <= d).sum())
+                tgt.ctx.verify_tree(tokens[:nd], parent[:nd], tgt.kv, tgt.logits.data_ptr())
+                for p in np.nonzero(depth == d)[0]:
+                    if not kids[int(p)]:
+                        continue
+                    g = 0.5 * torch.randn(V, device="cuda", generator=gen) ** 2      # Gamma(1/2) draws: a Dirichlet(1/2) row once normalised
+                    q = alpha * torch.softmax(tgt.logits[int(p)].double(), 0) + (1.0 - alpha) * (g / g.sum()).double()
+                    picks = torch.multinomial(q, len(kids[int(p)]), replacement=True, generator=gen).cpu().numpy()
+                    for c, t in zip(kids[int(p)], picks):
+                        tokens[c] = int(t)
+                        rows[c] = q.float()
+            # ---- timed: the target stage
+            ev[2].record(tgt.stream)
+            tgt.ctx.verify_tree(tokens, parent, tgt.kv, tgt.logits.data_ptr())
+            path0, next0 = tgt.ctx.accept_tree(tgt.logits.data_ptr(), rows.data_ptr(), tokens, parent, mode=ssd.SSD_SAMPLING, rng=srng)
+            tgt.ctx.kv_commit(tgt.kv, path0)
+            ev[3].record(tgt.stream)
+            torch.cuda.synchronize()
+            t_draft += ev[0].elapsed_time(ev[1])
+            t_target += ev[2].elapsed_time(ev[3])
+            new = [int(tokens[c]) for c in path0[1:]] + [int(next0)]
+            # (untimed) the draft's cache follows the emitted sequence
+            chain = np.asarray([root] + new[:-1], dtype=np.int32)
+            drf.ctx.verify_tree(chain, ssd_synth.tree_chain(len(chain)), drf.kv, dlogits.data_ptr())
+            drf.ctx.kv_commit(drf.kv, np.arange(len(chain), dtype=np.int32))
+            seq += new
+            emitted += len(new)
+            lengths.append(len(new))
+            steps += 1
+        method_ms = t_draft + t_target
+        out["alpha_%g" % alpha] = {
+            "emitted_tokens": emitted, "target_steps": steps, "tokens_per_target_step": emitted / steps,
+            "tokens_per_s": emitted / (method_ms * 1e-3), "us_per_step": {"draft_stage": t_draft * 1e3 / steps, "target_stage": t_target * 1e3 / steps},
+            "accepted_length_histogram": {str(k): int(lengths.count(k)) for k in sorted(set(lengths))}}
+    out["note"] = ("synthetic acceptance: proposal rows = alpha * softmax(target logits at the parent) + (1 - alpha) * Dirichlet(0.5), built by "
+                   "untimed level-by-level target forwards; timed = draft stage (2 rounds of trigram look-up, 8-node draft verify, acceptance, "
+                   "proposals, commit) + target stage (32-node verify, sampling acceptance, commit); prefix 64 growing with the emitted tokens")
+    tri.close()
+    tgt.close()
+    drf.close()
+    return out
+
+
 def run_gpu(args):
     import torch
 
@@ -495,6 +593,7 @@ def run_gpu(args):
             r2.close()
             del r2
         sweep.update(run_sweep(args, local, peaks))
+        sweep["config4"] = run_staged(args, local, peaks)
         line["sweep"] = sweep
     if world == 1 and not args.no_cpu_baseline:
         times = oracle_steps(cfg, weights, parent, P, np.random.default_rng(7), 3, 0, 60.0)
