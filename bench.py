@@ -528,7 +528,7 @@ def run_gpu(args):
     run = Runner(args.model, P, local, args.tune, rng_seed=1002 + rank)
     sampling = (args.temperature, args.top_k) if args.accept == "sampling" else None
     draft = torch.from_numpy(ssd_synth.draft_rows_gamma(n, run.V, run.rng)).cuda() if sampling else None
-    token_sets = run.planted_tokens(parent, 8, PLANT_PROBABILITY)
+    token_sets = run.planted_tokens(parent, args.plant_sets, PLANT_PROBABILITY)
 
     def barrier():
         if world > 1:
@@ -614,6 +614,7 @@ def main():
     ap.add_argument("--ref-budget-s", type=float, default=150.0)
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-sweep", action="store_true", help="skip the other configurations (16 / 64 nodes, draft model, XL sweep)")
+    ap.add_argument("--plant-sets", type=int, default=8, help="token sets prepared before the timed region (fewer = fewer launches before it, for profiling)")
     ap.add_argument("--tune", action="append", default=[], help="knob=value for ssd_set_tuning (experiments)")
     ap.add_argument("--accept", default="greedy", choices=["greedy", "sampling"],
                     help="acceptance rule of the step (the metric's workload is greedy; sampling draws draft rows from a Dirichlet)")
