@@ -48,7 +48,7 @@ NOMINAL_HBM_GBS = 8000.0
 PLANT_PROBABILITY = 0.6
 # DRAM bytes (read + write) of one forward of the metric's workload: sum over the ncu launch list in
 # profiles/bench_step_gpt2_large_n32_launch_list.md (per forward, like `achieved`)
-NCU_TRAFFIC_BYTES = {("gpt2_large", 32, 256): 1743.4e6}
+NCU_TRAFFIC_BYTES = {("gpt2_large", 32, 256): 1758.2e6}
 
 
 def measured_peaks():
