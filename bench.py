@@ -337,7 +337,7 @@ def per_kernel_roofline(run: Runner, parent, tokens, peak_gbs):
     cfg = run.cfg
     L, d, F, V = cfg["n_layer"], cfg["d_model"], cfg["d_ff"], cfg["vocab"]
     t = run.kernel_timeline(parent, tokens)
-    setup = 3
+    setup = 3  # tree preparation, clearing of the logits and embedding are not traced
     per = (len(t) - setup - 2) // L
     if per not in (5, 8) or len(t) != setup + per * L + 2:
         return None

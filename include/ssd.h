@@ -148,6 +148,9 @@ int ssd_verify_tree(ssd_ctx *ctx, const int32_t *tokens, const int32_t *parent_i
  * [n_nodes rounded up to 32, vocab] fp64 (plus 4 KB per node) of device scratch owned by the context (every node's target law
  * and the decision taken at it are computed side by side, then the walk follows the decisions); if that allocation fails the call still succeeds, computing the visited
  * rows one after the other.
+ * Deterministic mode on a bf16 model with SSD_TUNE_HEAD_STATS set: if `logits` is the buffer the context's last ssd_verify_tree wrote (same n_nodes), the walk
+ * reads the row maxima the LM head left per vocabulary tile instead of the logits themselves; do not modify that buffer between
+ * the two calls (or pass a copy: any other buffer is read in full).
  */
 int ssd_accept_tree(ssd_ctx *ctx, const float *logits, const float *draft_probs, const int32_t *tokens,
                     const int32_t *parent_idx, int32_t n_nodes, const ssd_sampling *sampling, ssd_rng *rng_state,
@@ -239,11 +242,17 @@ int ssd_kv_read(ssd_ctx *ctx, const ssd_kv *kv, int32_t layer, int32_t which, in
  *   SSD_TUNE_CLUSTER_MAX [8]      largest cluster (CTAs per output tile) of that path, 1..16
  *   SSD_TUNE_CLUSTER_QKV / _O / _FC / _PROJ [0]  cluster size of one of the four projections of a layer; 0 = choose
  *   SSD_TUNE_HEAD_CTAS [0]        CTAs of the LM-head projection; 0 = as the layers'
+ *   SSD_TUNE_HEAD_STATS [0]       the LM head runs one CTA per 128-word tile of the vocabulary over the whole width (complete sums,
+ *                                 plain stores, no clearing of the logits) and leaves per (row, tile) the maximum, its lowest index
+ *                                 and a non-finite flag; a greedy ssd_accept_tree on the buffer the last ssd_verify_tree of the
+ *                                 context wrote (same n_nodes, buffer not modified in between) reads those instead of the logits.
+ *                                 Measured: the forward 10 us slower (393 tiles over 296 CTA slots leave a ragged last wave), the
+ *                                 acceptance 10 us faster.  0 = stream-K head adding partial sums at L2 into cleared logits
  *   SSD_TUNE_KERNEL_TRACE [0]     record a timeline of every kernel of a bf16 forward (see ssd_get_phase_trace)
  */
 enum { SSD_TUNE_LOW_PLANE = 0, SSD_TUNE_DEPENDENT_LAUNCH = 1, SSD_TUNE_GRAPH = 2, SSD_TUNE_GEMM_CTAS = 3, SSD_TUNE_CLUSTER_REDUCE = 4,
        SSD_TUNE_CLUSTER_MAX = 5, SSD_TUNE_ATTN_LOW_PLANE = 6, SSD_TUNE_HEAD_CTAS = 7, SSD_TUNE_KERNEL_TRACE = 8, SSD_TUNE_CLUSTER_QKV = 9, SSD_TUNE_CLUSTER_O = 10,
-       SSD_TUNE_CLUSTER_FC = 11, SSD_TUNE_CLUSTER_PROJ = 12 };
+       SSD_TUNE_CLUSTER_FC = 11, SSD_TUNE_CLUSTER_PROJ = 12, SSD_TUNE_HEAD_STATS = 13 };
 int ssd_set_tuning(ssd_ctx *ctx, int32_t knob, int32_t value);
 
 /*

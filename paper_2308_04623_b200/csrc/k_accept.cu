@@ -67,29 +67,41 @@ __global__ void __launch_bounds__(256) row_argmax_kernel(const float *__restrict
     }
 }
 
-// The walk; a row's arg-max is the best of its `parts` parts (the parts are in index order, so the first one that
-// attains the maximum holds the lowest index).  `result` may be pinned host memory.
+// The walk, by one warp; a row's arg-max is the best of its `parts` parts (the parts are in index order, so among equal
+// maxima the lowest part holds the lowest index): the lanes take the parts round-robin.  `result` may be pinned host memory.
 __global__ void greedy_walk_kernel(NodeList tokens, NodeList parent, int n, int parts, const float *__restrict__ part_val,
                                    const int32_t *__restrict__ part_arg, const int32_t *__restrict__ part_bad, int32_t *__restrict__ result,
                                    const int32_t *__restrict__ dev_status) {
-    if (threadIdx.x != 0) return;
+    const int lane = threadIdx.x;
     int cur = 0, np = 1;
-    result[3] = dev_status ? *dev_status : 0; // the forward's error word rides along with the walk's few result words
-    result[4] = 0;
+    if (lane == 0) {
+        result[3] = dev_status ? *dev_status : 0; // the forward's error word rides along with the walk's few result words
+        result[4] = 0;
+    }
     for (;;) {
         float best = -INFINITY;
         int want = 0x7fffffff, bad = 0;
-        for (int q = 0; q < parts; ++q) {
-            const int at = cur * parts + q;
+        for (int q = lane; q < parts; q += 32) {
+            const size_t at = (size_t)cur * parts + q;
             bad |= part_bad[at];
-            if (part_val[at] > best || (part_val[at] == best && part_arg[at] < want)) { best = part_val[at]; want = part_arg[at]; }
+            const float v = part_val[at];
+            const int a = part_arg[at];
+            if (v > best || (v == best && a < want)) { best = v; want = a; }
         }
-        if (bad) { result[1] = -1; result[2] = SSD_ERR_BAD_ARG; result[0] = 1; return; }
+#pragma unroll
+        for (int off = 16; off > 0; off >>= 1) {
+            const float ov = __shfl_xor_sync(0xffffffffu, best, off);
+            const int oa = __shfl_xor_sync(0xffffffffu, want, off);
+            bad |= __shfl_xor_sync(0xffffffffu, bad, off);
+            if (ov > best || (ov == best && oa < want)) { best = ov; want = oa; }
+        }
+        if (bad) { if (lane == 0) { result[1] = -1; result[2] = SSD_ERR_BAD_ARG; result[0] = 1; } return; }
         int next = -1;
-        for (int c = cur + 1; c < n; ++c)
-            if (parent.v[c] == cur && tokens.v[c] == want) { next = c; break; }
-        if (next < 0) { result[1] = want; result[2] = SSD_OK; result[0] = np; return; }
-        result[4 + np++] = next;
+        for (int c = cur + 1; c < n && next < 0; ++c) // (the same scan in every lane)
+            if (parent.v[c] == cur && tokens.v[c] == want) next = c;
+        if (next < 0) { if (lane == 0) { result[1] = want; result[2] = SSD_OK; result[0] = np; } return; }
+        if (lane == 0) result[4 + np] = next;
+        ++np;
         cur = next;
     }
 }
@@ -419,10 +431,15 @@ cudaError_t launch_accept(const float *logits, const float *draft_probs, const N
                           int vocab, int mode, float temperature, int top_k, uint64_t seed, uint64_t step,
                           const AcceptScratch &sc, cudaStream_t s, int *launches) {
     if (mode == SSD_GREEDY) {
-        const int parts = sc.arg_parts > 0 ? sc.arg_parts : 1;
-        row_argmax_kernel<<<dim3(n, parts), 256, 0, s>>>(logits, vocab, sc.row_val, sc.row_arg, sc.row_bad);
-        greedy_walk_kernel<<<1, 32, 0, s>>>(tokens, parent, n, parts, sc.row_val, sc.row_arg, sc.row_bad, sc.result, sc.dev_status);
-        *launches += 2;
+        if (sc.head_parts > 0) { // the LM head left the rows' statistics per output tile: nothing of the logits is read again
+            greedy_walk_kernel<<<1, 32, 0, s>>>(tokens, parent, n, sc.head_parts, sc.head_val, sc.head_arg, sc.head_bad, sc.result, sc.dev_status);
+            *launches += 1;
+        } else {
+            const int parts = sc.arg_parts > 0 ? sc.arg_parts : 1;
+            row_argmax_kernel<<<dim3(n, parts), 256, 0, s>>>(logits, vocab, sc.row_val, sc.row_arg, sc.row_bad);
+            greedy_walk_kernel<<<1, 32, 0, s>>>(tokens, parent, n, parts, sc.row_val, sc.row_arg, sc.row_bad, sc.result, sc.dev_status);
+            *launches += 2;
+        }
     } else {
         double *rows = (sc.rows && sc.rows_cap >= n && n > 1) ? sc.rows : nullptr;
         if (rows) {
@@ -573,6 +590,7 @@ cudaError_t noalloc_setup(int device, AcceptScratch *out) {
         slot.sc.row_bad = (int32_t *)bad;
         slot.sc.result = (int32_t *)res;
         slot.sc.dev_status = nullptr;
+        slot.sc.head_parts = 0;
         slot.ready = true;
     }
     *out = slot.sc;

@@ -39,7 +39,7 @@ constexpr int UMMA_K = 16;                  // k per tcgen05.mma for 16-bit inpu
 constexpr int A_BYTES = TILE_M * TILE_K * 2;  // 16 KB
 constexpr int MAX_STAGES = 12;
 constexpr int GEMM_THREADS = 192;
-constexpr int SMEM_BUDGET = 220 * 1024;
+constexpr int SMEM_BUDGET = 210 * 1024;   // stages of one CTA per SM (the barriers and the statistics scratch follow them)
 constexpr int SMEM_BUDGET_SHARED = 106 * 1024;
 #ifndef EPI_POLL_NS
 #define EPI_POLL_NS 32
@@ -57,10 +57,18 @@ struct GemmParams {
     int split;         // > 0: every output tile's k tiles are shared by `split` CTAs of its own (grid = split * n_tiles); 0: stream-K ranges
     int use_lo;
     int32_t *status;   // device error word
+    // LM head with complete sums (split == 1): plain stores instead of reductions, and per (row, output tile) the maximum,
+    // its lowest index and a non-finite flag, so that greedy acceptance need not read the logits again
+    int store;
+    float *stat_val;   // [n, n_tiles] or null
+    int32_t *stat_arg, *stat_bad;
     unsigned long long *trace; // timeline slots of this launch or null
 };
 
 struct __align__(8) Barriers {
+    float stat_val[4][SSD_MAX_NODES];   // the four epilogue warps' row maxima over their 32 features (statistics epilogue)
+    int32_t stat_arg[4][SSD_MAX_NODES];
+    int32_t stat_bad[4];
     uint64_t full[MAX_STAGES];
     uint64_t empty[MAX_STAGES];
     uint64_t acc_full[2];
@@ -241,12 +249,38 @@ gemm_ws_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant_
             if (!good) { if (lane == 0) fail(p, bars, 0x400 + ab); ok = false; }
             if (seg == 0 && et == 0) ptx::trace_mark(p.trace, 3); // first accumulator complete
             ptx::tc_fence_after_sync();
+            int warp_bad = 0;
             for (int c0 = 0; c0 < p.n_pad && good; c0 += 16) {
                 uint32_t r[16], q[16];
                 ptx::tmem_ld_32x16(taddr + c0, r);
                 if (stacked) ptx::tmem_ld_32x16(taddr + p.n_pad + c0, q); // the lo plane's part of the product
                 ptx::tmem_ld_wait();
-                if (o < p.out) {
+                if (p.store) { // this CTA holds the complete sums of its tile: plain stores, and the rows' statistics over the tile
+                    float v[16];
+#pragma unroll
+                    for (int t = 0; t < 16; ++t) {
+                        v[t] = __uint_as_float(r[t]) + (stacked ? __uint_as_float(q[t]) : 0.f) + bias;
+                        if (o < p.out && c0 + t < p.n) y[(size_t)(c0 + t) * p.ldy + o] = v[t];
+                    }
+                    if (p.stat_val) {
+                        // row maximum over this warp's 32 features with one warp-wide integer reduction per row: floats map to
+                        // unsigned keys of the same order; the lowest lane holding the maximum is the lowest index
+#pragma unroll
+                        for (int t = 0; t < 16; ++t) {
+                            const bool live = o < p.out;
+                            warp_bad |= (live && c0 + t < p.n && !isfinite(v[t])) ? 1 : 0;
+                            const unsigned bits = __float_as_uint(v[t]);
+                            unsigned key = (bits & 0x80000000u) ? ~bits : (bits | 0x80000000u);
+                            if (!live || v[t] != v[t]) key = 0u;       // (padding features and NaNs never win; the flag reports NaNs)
+                            const unsigned top = __reduce_max_sync(0xffffffffu, key);
+                            const unsigned who = __ballot_sync(0xffffffffu, key == top);
+                            if (lane == 0 && c0 + t < p.n) {
+                                bars->stat_val[quarter][c0 + t] = top == 0u ? -INFINITY : __uint_as_float((top & 0x80000000u) ? (top & 0x7fffffffu) : ~top);
+                                bars->stat_arg[quarter][c0 + t] = tile * TILE_M + quarter * 32 + (__ffs(who) - 1);
+                            }
+                        }
+                    }
+                } else if (o < p.out) {
                     float *yo = y + (size_t)c0 * p.ldy + o;
                     if (stacked && c0 + 16 <= p.n) { // the usual case, kept short: sixteen full rows, hi + lo columns
 #pragma unroll
@@ -262,6 +296,23 @@ gemm_ws_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant_
                         }
                     }
                 }
+            }
+            if (p.store && p.stat_val) { // the four warps' 32-feature shares -> one (maximum, lowest index, flag) per row and tile
+                warp_bad = __any_sync(0xffffffffu, warp_bad);
+                if (lane == 0) bars->stat_bad[quarter] = warp_bad;
+                epi_sync();
+                for (int i = et; i < p.n; i += 128) {
+                    float best = bars->stat_val[0][i];
+                    int arg = bars->stat_arg[0][i];
+#pragma unroll
+                    for (int w = 1; w < 4; ++w)
+                        if (bars->stat_val[w][i] > best || (bars->stat_val[w][i] == best && bars->stat_arg[w][i] < arg)) { best = bars->stat_val[w][i]; arg = bars->stat_arg[w][i]; }
+                    const size_t at = (size_t)i * p.n_tiles + tile;
+                    p.stat_val[at] = good ? best : -INFINITY;
+                    p.stat_arg[at] = arg;
+                    p.stat_bad[at] = (bars->stat_bad[0] | bars->stat_bad[1] | bars->stat_bad[2] | bars->stat_bad[3]) ? 1 : 0;
+                }
+                epi_sync();
             }
             ptx::tc_fence_before_sync();
             __syncwarp();
@@ -327,12 +378,13 @@ cudaError_t gemm_ws_prepare() {
 
 cudaError_t launch_gemm_ws(const void *map_w, const void *map_hi, const void *map_lo, float *y, const StepInfo *info, int ldy,
                            const float *bias, int n, int K, int out, int use_lo, int grid, int sm_count, int32_t *status, bool pdl,
-                           cudaStream_t s, unsigned long long *trace) {
+                           cudaStream_t s, unsigned long long *trace, const GemmHeadStats *head) {
     GemmParams p;
     p.trace = trace;
     p.y = y; p.info = info; p.bias = bias; p.n = n; p.n_pad = (n + 15) & ~15;
     p.out = out; p.ldy = ldy; p.k_tiles = K / TILE_K; p.n_tiles = (out + TILE_M - 1) / TILE_M;
     p.use_lo = use_lo; p.status = status;
+    p.store = 0; p.stat_val = nullptr; p.stat_arg = nullptr; p.stat_bad = nullptr;
     const int stage_bytes = A_BYTES + p.n_pad * TILE_K * 2 * (use_lo ? 2 : 1);
     const long long units = (long long)p.n_tiles * p.k_tiles;
     if (grid > units) grid = (int)units;
@@ -349,6 +401,10 @@ cudaError_t launch_gemm_ws(const void *map_w, const void *map_hi, const void *ma
         if (p.n_pad >= 64 && per_cta < 2 && p.k_tiles >= 2) per_cta = 2;
         p.split = (p.k_tiles + per_cta - 1) / per_cta;          // ... and the fewest CTAs per tile that reach it
         grid = p.split * p.n_tiles;
+    }
+    if (head) { // complete sums: one CTA per output tile, whatever the grid asked for
+        p.split = 1; grid = p.n_tiles; per_cta = p.k_tiles;
+        p.store = 1; p.stat_val = head->val; p.stat_arg = head->arg; p.stat_bad = head->bad;
     }
     p.stages = gemm_ws_stages(p.n_pad, use_lo, grid > sm_count);
     if (p.stages > per_cta) p.stages = per_cta < 1 ? 1 : per_cta;

@@ -65,6 +65,12 @@ struct ssd_ctx {
     float *d_sparse_val, *d_sparse_rows;
     size_t sparse_entries_cap, sparse_rows_cap;
     int32_t *d_status;
+    // per (row, output tile) statistics of the logits, written by the LM head (bf16 path), and which logits buffer they describe
+    float *head_val;
+    int32_t *head_arg, *head_bad;
+    int head_tiles, use_head_stats;
+    const float *head_logits;
+    int head_n;
 };
 
 namespace {
@@ -197,7 +203,11 @@ cudaError_t enqueue_forward(ssd_ctx *ctx, int n, int cap, const NodeList &tk, co
     cudaError_t e;
 #define Q(call) do { if ((e = (call)) != cudaSuccess) return e; ++*kernels; } while (0)
     Q(launch_tree_prep(tk, pr, step, ctx->meta, ctx->d_info, s));
-    if (ctx->tensor_path) Q(launch_zero_logits(info, n, c.vocab, s)); // the LM head adds its stream-K partial sums into them
+    // The LM head either holds complete sums per CTA (plain stores, row statistics per tile) or adds stream-K partial sums
+    // into logits cleared here, at the start of the forward.
+    const GemmHeadStats head_stats = {ctx->head_val, ctx->head_arg, ctx->head_bad};
+    const GemmHeadStats *head = (ctx->tensor_path && ctx->use_head_stats) ? &head_stats : nullptr;
+    if (ctx->tensor_path && !head) Q(launch_zero_logits(info, n, c.vocab, s));
     if (ctx->tensor_path && ctx->use_cluster && gemm_cl_supports(n, c.d_model)) {
         // bf16 model, trees of up to 64 nodes: five launches per layer.  Every projection reduces its split-K partial sums
         // inside a thread-block cluster, so its epilogue holds finished sums and does the work that would otherwise be
@@ -243,7 +253,7 @@ cudaError_t enqueue_forward(ssd_ctx *ctx, int n, int cap, const NodeList &tk, co
         }
         const int hgrid = head_grid_for(ctx, n);
         Q(launch_ln_prep(ctx->x, ctx->lnf_g, ctx->lnf_b, n, d, c.ln_eps, ctx->a_hi, a_lo, nullptr, 0, info, 0, pdl, s, trace_slot(ctx, *kernels)));
-        Q(launch_gemm_ws(&ctx->map_wte, &amh->a_hi, &amh->a_lo, nullptr, info, c.vocab, nullptr, n, d, c.vocab, lo, hgrid, sms, ctx->d_status, pdl, s, trace_slot(ctx, *kernels)));
+        Q(launch_gemm_ws(&ctx->map_wte, &amh->a_hi, &amh->a_lo, nullptr, info, c.vocab, nullptr, n, d, c.vocab, lo, hgrid, sms, ctx->d_status, pdl, s, trace_slot(ctx, *kernels), head));
         ctx->trace_count = ctx->trace_kernels ? 8 * *kernels : 0;
         return cudaSuccess;
     }
@@ -267,7 +277,7 @@ cudaError_t enqueue_forward(ssd_ctx *ctx, int n, int cap, const NodeList &tk, co
             Q(launch_gemm_ws(&t[3], &am->h_hi, &am->h_lo, ctx->x, info, d, L.b_proj, n, F, d, lo, grid, sms, ctx->d_status, pdl, s, trace_slot(ctx, *kernels)));
         }
         Q(launch_ln_prep(ctx->x, ctx->lnf_g, ctx->lnf_b, n, d, c.ln_eps, ctx->a_hi, a_lo, nullptr, 0, info, 0, pdl, s, trace_slot(ctx, *kernels)));
-        Q(launch_gemm_ws(&ctx->map_wte, &am->a_hi, &am->a_lo, nullptr, info, c.vocab, nullptr, n, d, c.vocab, lo, hgrid, sms, ctx->d_status, pdl, s, trace_slot(ctx, *kernels)));
+        Q(launch_gemm_ws(&ctx->map_wte, &am->a_hi, &am->a_lo, nullptr, info, c.vocab, nullptr, n, d, c.vocab, lo, hgrid, sms, ctx->d_status, pdl, s, trace_slot(ctx, *kernels), head));
         ctx->trace_count = ctx->trace_kernels ? 8 * *kernels : 0;
     } else {
         for (int l = 0; l < c.n_layer; ++l) {
@@ -393,6 +403,9 @@ int ssd_create(const ssd_config *cfg, int device, void *cuda_stream, ssd_ctx **o
     A(&ctx->x, n * d); A(&ctx->a, n * d); A(&ctx->qkv, n * 3 * d); A(&ctx->o, n * d); A(&ctx->h, n * (size_t)cfg->d_ff);
     ctx->acc.arg_parts = 4;
     ctx->acc.dev_status = nullptr;
+    ctx->acc.head_parts = 0;
+    ctx->head_val = nullptr; ctx->head_arg = ctx->head_bad = nullptr; ctx->head_tiles = 0; ctx->use_head_stats = 0;
+    ctx->head_logits = nullptr; ctx->head_n = 0;
     A(&ctx->acc.r, (size_t)cfg->vocab); A(&ctx->acc.row_val, 4 * n); A(&ctx->acc.row_arg, 4 * n); A(&ctx->acc.row_bad, 4 * n); A(&ctx->acc.result, n + 4);
     A(&ctx->d_status, 1);
     A(&ctx->d_info, 1);
@@ -418,6 +431,8 @@ int ssd_create(const ssd_config *cfg, int device, void *cuda_stream, ssd_ctx **o
         const size_t rows = n <= 32 ? 32 : ((n + 15) & ~size_t(15)); // operand planes hold whole 16-row boxes, at least two
         A(&ctx->a_hi, rows * d); A(&ctx->a_lo, rows * d); A(&ctx->o_hi, rows * d); A(&ctx->o_lo, rows * d);
         A(&ctx->h_hi, rows * (size_t)cfg->d_ff); A(&ctx->h_lo, rows * (size_t)cfg->d_ff);
+        ctx->head_tiles = (cfg->vocab + 127) / 128;
+        A(&ctx->head_val, n * (size_t)ctx->head_tiles); A(&ctx->head_arg, n * (size_t)ctx->head_tiles); A(&ctx->head_bad, n * (size_t)ctx->head_tiles);
         if (rc == SSD_OK) {
             cudaError_t e = cudaSuccess;
             __nv_bfloat16 *planes[6] = {ctx->a_hi, ctx->a_lo, ctx->o_hi, ctx->o_lo, ctx->h_hi, ctx->h_lo};
@@ -627,6 +642,8 @@ int ssd_verify_tree(ssd_ctx *ctx, const int32_t *tokens, const int32_t *parent_i
         CU(enqueue_forward(ctx, n_nodes, kv->cap, tk, pr, step, ctx->stream, &kernels));
     }
     ctx->launches += kernels;
+    ctx->head_logits = (ctx->tensor_path && ctx->use_head_stats) ? logits_out : nullptr;
+    ctx->head_n = n_nodes;
     kv->last_n = n_nodes;
     memcpy(kv->last_parent, parent_idx, sizeof(int32_t) * n_nodes);
     return SSD_OK;
@@ -658,6 +675,10 @@ int ssd_accept_tree(ssd_ctx *ctx, const float *logits, const float *draft_probs,
     AcceptScratch sc = ctx->acc;
     sc.result = ctx->h_result; // the walk writes its few words straight into the pinned host buffer: no copy to enqueue and wait for
     sc.dev_status = ctx->d_status;
+    // greedy on the very logits the last forward of this context wrote: the LM head's per-tile row statistics stand in for them
+    if (sampling->mode == SSD_GREEDY && ctx->head_logits && ctx->head_logits == logits && ctx->head_n == n) {
+        sc.head_parts = ctx->head_tiles; sc.head_val = ctx->head_val; sc.head_arg = ctx->head_arg; sc.head_bad = ctx->head_bad;
+    }
     ctx->h_result[0] = 0;
     CU(launch_accept(logits, draft_probs, tk, pr, n, c.vocab, sampling->mode, sampling->temperature, sampling->top_k, rng_state->seed,
                      rng_state->step, sc, ctx->stream, &launched));
@@ -804,6 +825,7 @@ int ssd_set_tuning(ssd_ctx *ctx, int32_t knob, int32_t value) {
     case SSD_TUNE_HEAD_CTAS: if (value < 0 || value > 4096) return SSD_ERR_BAD_ARG; ctx->head_grid = value; break;
     case SSD_TUNE_CLUSTER_REDUCE: if (value != 0 && value != 1) return SSD_ERR_BAD_ARG; ctx->use_cluster = value; break;
     case SSD_TUNE_ATTN_LOW_PLANE: if (value != 0 && value != 1) return SSD_ERR_BAD_ARG; ctx->attn_lo = value; break;
+    case SSD_TUNE_HEAD_STATS: if (value != 0 && value != 1) return SSD_ERR_BAD_ARG; ctx->use_head_stats = value; ctx->head_logits = nullptr; break;
     case SSD_TUNE_CLUSTER_MAX: if (value < 1 || value > 16) return SSD_ERR_BAD_ARG; ctx->cl_max = value; break;
     case SSD_TUNE_CLUSTER_QKV: case SSD_TUNE_CLUSTER_O: case SSD_TUNE_CLUSTER_FC: case SSD_TUNE_CLUSTER_PROJ:
         if (value < 0 || value > 16) return SSD_ERR_BAD_ARG;

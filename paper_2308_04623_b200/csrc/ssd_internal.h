@@ -78,9 +78,12 @@ cudaError_t prep_kernels_prepare();
 // activation planes [rows >= n_pad, K], ONE box of n_pad rows (map_lo may be null when use_lo = 0).
 // If y is null the destination is info->logits.  `grid` CTAs share the units; with grid > sm_count each takes at most
 // half an SM's shared memory.
+// With `head` set the projection runs one CTA per output tile over the whole K (complete sums): plain stores, no clearing of Y
+// needed, and per (row, tile) the maximum, its lowest feature index and a non-finite flag at [row * n_tiles + tile].
+struct GemmHeadStats { float *val; int32_t *arg, *bad; };
 cudaError_t launch_gemm_ws(const void *map_w, const void *map_hi, const void *map_lo, float *y, const StepInfo *info, int ldy,
                            const float *bias, int n, int K, int out, int use_lo, int grid, int sm_count, int32_t *status, bool pdl,
-                           cudaStream_t s, unsigned long long *trace = nullptr);
+                           cudaStream_t s, unsigned long long *trace = nullptr, const GemmHeadStats *head = nullptr);
 // ---- projection with the split-K sums reduced inside a thread-block cluster (trees of up to 64 nodes) ----
 // What the epilogue does with the finished sums acc[i, o] (see k_gemm_cl.cu):
 enum { MODE_FOLD_STORE = 0, MODE_FOLD_GELU = 1, MODE_RESIDUAL = 2 };
@@ -141,6 +144,10 @@ struct AcceptScratch {
     int32_t *row_bad;   // [max_nodes * parts] 1 if the part holds a non-finite value (sampling: [max_nodes], per row)
     int32_t *result;    // [max_nodes + 4]: n_path, next_token, status, device error word, path[...]
     const int32_t *dev_status; // the forward's device error word (copied into result[3] by the walk) or null
+    // greedy: per (row, part) statistics already written by the LM head (parts = head_parts > 0): the arg-max pass is skipped
+    int head_parts;
+    const float *head_val;
+    const int32_t *head_arg, *head_bad;
 };
 cudaError_t launch_propose_children(const float *logits, const NodeList &nodes, int m, int vocab, int mode, float temperature, int top_k, int picks,
                                     uint64_t seed, uint64_t step, double *scratch, float *rows_out, int32_t *tokens_out, int32_t *bad_out,

@@ -454,6 +454,7 @@ def test_bf16_steps_with_commit(util):
     import paper_2308_04623_b200 as ssd
     p = util.Pair("ragged_bf16", seed=2)
     try:
+        p.ctx.set_tuning(ssd.SSD_TUNE_HEAD_STATS, 1)  # (the LM head with complete sums and row statistics; the default head is tested everywhere else)
         rng = np.random.default_rng(3)
         p.prefill(ssd_synth.uniform_tokens(33, p.V, rng))
         root = 5
@@ -467,9 +468,15 @@ def test_bf16_steps_with_commit(util):
                 if rng.random() < 0.6:
                     tokens[c] = int(np.argmax(got[parent[c]]))
             got, want, buf = p.verify(tokens, parent)
+            launches = p.ctx.kernel_launches()
             path, nxt = p.ctx.accept_tree(buf.data_ptr(), None, tokens, parent, mode=ssd.SSD_GREEDY)
+            assert p.ctx.kernel_launches() - launches == 1    # the walk alone: the LM head left the rows' statistics per vocabulary tile
             opath, onxt, _ = ssd_oracle.accept_tree(got.astype(np.float32), None, tokens, parent, mode=0)
             assert (path, nxt) == (opath, onxt)
+            other = buf.clone()                               # the same logits in another buffer: the arg-max pass runs, same result
+            launches = p.ctx.kernel_launches()
+            assert p.ctx.accept_tree(other.data_ptr(), None, tokens, parent, mode=ssd.SSD_GREEDY) == (path, nxt)
+            assert p.ctx.kernel_launches() - launches == 2
             p.commit(path)
             root = nxt
             # committed rows: bf16 storage of the fp32 projections, compared with the oracle's exact rows
@@ -542,6 +549,38 @@ def test_projection_cta_counts_give_the_same_logits(ctas, util, ssd):
         tokens = ssd_synth.uniform_tokens(29, p.V, rng)
         got, want, _ = p.verify(tokens, parent)
         assert np.abs(got - want).max() <= TOL_BF16
+        assert p.ctx.device_status() == 0
+    finally:
+        p.close()
+
+
+@pytest.mark.parametrize("name,n", [("ragged_bf16", 29), ("tiny_bf16", 100)])
+def test_head_with_row_statistics_and_stream_k_head_give_the_same_logits(name, n, util, ssd):
+    """SSD_TUNE_HEAD_STATS = 1: the LM head with complete sums per CTA (plain stores, no clearing launch, per-tile row
+    maxima that the greedy walk reads instead of the logits) against the default stream-K head adding partial sums into
+    cleared logits, greedy acceptance with its own arg-max pass; same logits within reduction-order noise, same paths."""
+    p = util.Pair(name, seed=4, qk_gain=3.0)
+    try:
+        p.ctx.set_tuning(ssd.SSD_TUNE_HEAD_STATS, 1)
+        rng = np.random.default_rng(5)
+        p.prefill(ssd_synth.uniform_tokens(21, p.V, rng), chunk=16)
+        parent = ssd_synth.tree_random(n, 5, rng)
+        tokens = ssd_synth.uniform_tokens(n, p.V, rng)
+        got, want, buf = p.verify(tokens, parent)
+        assert np.abs(got - want).max() <= TOL_BF16
+        before = p.ctx.kernel_launches()
+        first = p.ctx.accept_tree(buf.data_ptr(), None, tokens, parent)
+        assert p.ctx.kernel_launches() - before == 1
+        p.ctx.set_tuning(ssd.SSD_TUNE_HEAD_STATS, 0)
+        before = p.ctx.kernel_launches()
+        plain, _, buf2 = p.verify(tokens, parent)
+        assert p.ctx.kernel_launches() - before == 3 + 8 * p.cfg["n_layer"] + 2
+        assert np.abs(plain - got).max() <= 1e-3 and np.abs(plain - want).max() <= TOL_BF16
+        before = p.ctx.kernel_launches()
+        opath, onxt, _ = ssd_oracle.accept_tree(plain.astype(np.float32), None, tokens, parent, mode=0)
+        assert p.ctx.accept_tree(buf2.data_ptr(), None, tokens, parent) == (opath, onxt)
+        assert p.ctx.kernel_launches() - before == 2
+        assert first == ssd_oracle.accept_tree(got.astype(np.float32), None, tokens, parent, mode=0)[:2]
         assert p.ctx.device_status() == 0
     finally:
         p.close()
