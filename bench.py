@@ -117,7 +117,7 @@ def tree_rule(n_nodes):
 
 
 def workload(args):
-    cfg = ssd_synth.config(args.model)
+    cfg = ssd_synth.config(args.model, dtype=getattr(args, "weights", "bf16"))
     parent = ssd_synth.tree_branching(args.nodes, tree_rule(args.nodes))
     return cfg, parent
 
@@ -233,17 +233,17 @@ def run_reference(args):
 class Runner:
     """One model on the device with a prefilled cache; times steps of a given tree."""
 
-    def __init__(self, model, prefix_len, device, tune=(), seed=0, rng_seed=1002):
+    def __init__(self, model, prefix_len, device, tune=(), seed=0, rng_seed=1002, dtype=None):
         import torch
         import paper_2308_04623_b200 as ssd
         self.torch, self.ssd = torch, ssd
-        self.cfg = ssd_synth.config(model)
+        self.cfg = ssd_synth.config(model, **({"dtype": dtype} if dtype else {}))
         self.model, self.P, self.V = model, prefix_len, self.cfg["vocab"]
         self.rng = np.random.default_rng(rng_seed)
         self.weights = ssd_synth.make_weights(self.cfg, seed=seed)
         self.stream = torch.cuda.current_stream()
         self.ctx = ssd.Context(self.cfg, device=device, stream=self.stream.cuda_stream)
-        self.ctx.load_weights(ssd_synth.bf16_bits(self.weights) if self.cfg["dtype"] == "bf16" else self.weights)
+        self.ctx.load_weights(ssd_synth.bf16_bits(self.weights) if self.cfg["dtype"] != "fp32" else self.weights)
         for spec in tune:
             knob, value = spec.split("=")
             self.ctx.set_tuning(int(knob), int(value))
@@ -345,7 +345,11 @@ def per_kernel_roofline(run: Runner, parent, tokens, peak_gbs):
     dur = (body[:, :, 6] - body[:, :, 1]) / 1e3  # dependencies met -> latest end, us
     med = np.median(dur[2:], axis=0)
     names = ["ln1", "qkv", "attention", "o_proj", "ln2", "fc", "gelu", "proj"] if per == 8 else ["qkv", "attention", "o_proj", "fc", "proj"]
-    weight_bytes = {"qkv": 2 * 3 * d * d, "o_proj": 2 * d * d, "fc": 2 * d * F, "proj": 2 * d * F}
+    mb = 1 if cfg["dtype"] == "bf16_w8" else 2   # bytes per matrix entry (8-bit codes carry 4 more bytes per output row)
+    rows_of = {"qkv": 3 * d, "o_proj": d, "fc": F, "proj": d}
+    weight_bytes = {"qkv": mb * 3 * d * d, "o_proj": mb * d * d, "fc": mb * d * F, "proj": mb * d * F}
+    if mb == 1:
+        weight_bytes = {k: v + 4 * rows_of[k] for k, v in weight_bytes.items()}
     out = {}
     for name, us in zip(names, med):
         e = {"us": float(us)}
@@ -355,7 +359,7 @@ def per_kernel_roofline(run: Runner, parent, tokens, peak_gbs):
             e["frac"] = e["achieved_gbs"] / peak_gbs
         out[name] = e
     head_us = float(t[-1, 6] - t[-1, 1]) / 1e3
-    head_bytes = 2 * V * d + 4 * len(parent) * V
+    head_bytes = mb * V * d + (4 * V if mb == 1 else 0) + 4 * len(parent) * V
     out["lm_head"] = {"us": head_us, "algorithmic_bytes": head_bytes, "achieved_gbs": head_bytes / (head_us * 1e-6) / 1e9,
                       "frac": head_bytes / (head_us * 1e-6) / 1e9 / peak_gbs}
     deps = body[:, 0, 1].astype(np.float64)
@@ -525,7 +529,7 @@ def run_gpu(args):
         dist.init_process_group("nccl", device_id=torch.device("cuda", local))
     cfg, parent = workload(args)
     n, P = len(parent), args.prefix
-    run = Runner(args.model, P, local, args.tune, rng_seed=1002 + rank)
+    run = Runner(args.model, P, local, args.tune, rng_seed=1002 + rank, dtype=args.weights)
     sampling = (args.temperature, args.top_k) if args.accept == "sampling" else None
     draft = torch.from_numpy(ssd_synth.draft_rows_gamma(n, run.V, run.rng)).cuda() if sampling else None
     token_sets = run.planted_tokens(parent, args.plant_sets, PLANT_PROBABILITY)
@@ -559,9 +563,9 @@ def run_gpu(args):
     line = {
         "metric": METRIC, "value": replica_value(ms_per_step, world), "unit": UNIT, "n_gpus": world, "steps": args.steps,
         "warmup": args.warmup, "ms_per_step": ms_per_step, "higher_is_better": False, "scaling": "weak", "vs_baseline": None,
-        "dtype": "bf16" if cfg["dtype"] == "bf16" else "f32", "data": "synthetic",
-        "config": {"workload": "%s verify n=%d prefix=%d, %s accept, commit" % (
-                       args.model, n, P, ("sampling (T=%g, top-k=%d)" % (args.temperature, args.top_k)) if sampling else "greedy"),
+        "dtype": "bf16" if cfg["dtype"] != "fp32" else "f32", "data": "synthetic",
+        "config": {"workload": "%s%s verify n=%d prefix=%d, %s accept, commit" % (
+                       args.model, " (matrices as 8-bit codes)" if cfg["dtype"] == "bf16_w8" else "", n, P, ("sampling (T=%g, top-k=%d)" % (args.temperature, args.top_k)) if sampling else "greedy"),
                    "tree": "branching %s BFS truncated at %d" % (list(tree_rule(n)), n),
                    "tokens": "uniform ids, the verifier's arg-max planted on each child with probability %g" % PLANT_PROBABILITY,
                    "l2": "inputs larger than L2 (%.0f MB of weights per step)" % (alg_bytes / 1e6), "replicas": world,
@@ -615,6 +619,8 @@ def main():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-sweep", action="store_true", help="skip the other configurations (16 / 64 nodes, draft model, XL sweep)")
     ap.add_argument("--plant-sets", type=int, default=8, help="token sets prepared before the timed region (fewer = fewer launches before it, for profiling)")
+    ap.add_argument("--weights", default="bf16", choices=["bf16", "bf16_w8"],
+                    help="how the library holds the matrices it streams: bf16 (the benchmark's configuration) or 8-bit codes with per-row scales")
     ap.add_argument("--tune", action="append", default=[], help="knob=value for ssd_set_tuning (experiments)")
     ap.add_argument("--accept", default="greedy", choices=["greedy", "sampling"],
                     help="acceptance rule of the step (the metric's workload is greedy; sampling draws draft rows from a Dirichlet)")

@@ -51,11 +51,21 @@ enum {
 
 typedef struct {
     int32_t n_layer, d_model, n_head, d_head, d_ff, vocab, n_ctx, max_nodes;
-    int32_t dtype; /* 0: fp32 weights and cache; 1: bf16 weights and cache, fp32 accumulation */
+    int32_t dtype; /* 0: fp32 weights and cache; 1: bf16 weights and cache, fp32 accumulation; 2: as 1 with 8-bit matrices */
     float ln_eps;
 } ssd_config;
 
-enum { SSD_DTYPE_F32 = 0, SSD_DTYPE_BF16 = 1 };
+/*
+ * SSD_DTYPE_BF16_W8 (8-bit quantisation is the second item of the future-work list that closes Section 4): the model is
+ * given and run as the bf16 model, but ssd_load_weights re-encodes the matrices the projections stream - w_qkv, w_o,
+ * w_fc, w_proj and the output head (wte) - as e4m3 codes (1 sign, 4 exponent, 3 fraction bits) with one fp32 scale per
+ * output row, halving the bytes a step reads.  The scale of a row is the smallest power of two s with max|w| <= 448 s
+ * (1 for a row of zeros); code = round-to-nearest-even(w / s), saturating; the kernels compute with code * s exactly
+ * (the codes are widened to bf16 on chip, the scale multiplies the fp32 sums).  A matrix whose entries are already
+ * code * power-of-two values is therefore represented without loss.  The embedding look-up keeps the bf16 table;
+ * biases, LayerNorm parameters, activations and the cache are as with dtype 1.
+ */
+enum { SSD_DTYPE_F32 = 0, SSD_DTYPE_BF16 = 1, SSD_DTYPE_BF16_W8 = 2 };
 enum { SSD_GREEDY = 0, SSD_SAMPLING = 1 };
 
 typedef struct {
@@ -72,7 +82,7 @@ typedef struct {
 
 /* Host pointers to the model in its plain layout.  Every matrix is [out_features, in_features]
  * row-major; w_qkv stacks query, key and value rows (each head-major).  Elements are float when
- * dtype = 0 and bf16 bit patterns (uint16_t) when dtype = 1 - LayerNorm gains/biases and linear
+ * dtype = 0 and bf16 bit patterns (uint16_t) when dtype = 1 or 2 - LayerNorm gains/biases and linear
  * biases included.  Per-layer members are arrays of n_layer pointers. */
 typedef struct {
     const void *wte;   /* [vocab, d_model] token embedding, also the output head */
@@ -100,6 +110,15 @@ int ssd_create(const ssd_config *cfg, int device, void *cuda_stream, ssd_ctx **o
  * any verify call.  Synchronises the stream.
  */
 int ssd_load_weights(ssd_ctx *ctx, const ssd_weights *w);
+
+/*
+ * Read back one 8-bit matrix of a SSD_DTYPE_BF16_W8 context (to check the encoding): which = 0 w_qkv, 1 w_o, 2 w_fc,
+ * 3 w_proj of layer `layer`, 4 the output head (layer ignored).
+ *   codes_out  : host, [rows, cols] bytes (e4m3 bit patterns), rows / cols those of the matrix
+ *   scales_out : host, [rows] float
+ * Errors: BAD_ARG (also for a context of another dtype), NOT_LOADED, CUDA.  Synchronises the stream.
+ */
+int ssd_w8_read(ssd_ctx *ctx, int32_t which, int32_t layer, uint8_t *codes_out, float *scales_out);
 
 /* Cache objects.  A new or reset cache has length 0.  Rollback shortens the committed length
  * (len <= current length); rows above the length are scratch and may be overwritten. */

@@ -12,12 +12,13 @@ _LIB_PATH = os.path.join(_HERE, "libssd.so")
 SSD_OK, SSD_ERR_BAD_ARG, SSD_ERR_NOT_LOADED, SSD_ERR_INVALID_TREE, SSD_ERR_CTX_OVERFLOW = 0, -1, -2, -3, -4
 SSD_ERR_BAD_PATH, SSD_ERR_CUDA, SSD_ERR_TIMEOUT, SSD_ERR_NOMEM, SSD_ERR_UNSUPPORTED = -5, -6, -7, -8, -9
 SSD_GREEDY, SSD_SAMPLING = 0, 1
+SSD_DTYPE_F32, SSD_DTYPE_BF16, SSD_DTYPE_BF16_W8 = 0, 1, 2
 SSD_TUNE_LOW_PLANE, SSD_TUNE_DEPENDENT_LAUNCH, SSD_TUNE_GRAPH, SSD_TUNE_GEMM_CTAS, SSD_TUNE_CLUSTER_REDUCE, SSD_TUNE_CLUSTER_MAX = 0, 1, 2, 3, 4, 5
 SSD_TUNE_ATTN_LOW_PLANE, SSD_TUNE_HEAD_CTAS, SSD_TUNE_KERNEL_TRACE = 6, 7, 8
 SSD_TUNE_CLUSTER_QKV, SSD_TUNE_CLUSTER_O, SSD_TUNE_CLUSTER_FC, SSD_TUNE_CLUSTER_PROJ, SSD_TUNE_HEAD_STATS = 9, 10, 11, 12, 13
 
 # every symbol include/ssd.h declares
-EXPORTS = ("ssd_create", "ssd_load_weights", "ssd_kv_create", "ssd_kv_reset", "ssd_kv_len", "ssd_kv_rollback",
+EXPORTS = ("ssd_create", "ssd_load_weights", "ssd_w8_read", "ssd_kv_create", "ssd_kv_reset", "ssd_kv_len", "ssd_kv_rollback",
            "ssd_kv_destroy", "ssd_verify_tree", "ssd_accept_tree", "ssd_accept_tree_sparse", "ssd_propose_children", "ssd_kv_commit", "ssd_kv_read", "ssd_strerror",
            "ssd_last_device_status", "ssd_reset_device_status", "ssd_debug_expire_wait", "ssd_last_cuda_error", "ssd_last_cuda_error_line", "ssd_kernel_launches", "ssd_set_tuning", "ssd_get_phase_trace", "ssd_accept_tree_noalloc", "ssd_destroy",
            "ssd_trigram_build", "ssd_trigram_lookup", "ssd_trigram_propose", "ssd_trigram_contexts", "ssd_trigram_destroy")
@@ -62,6 +63,7 @@ def lib():
         L = C.CDLL(_LIB_PATH)
         L.ssd_create.argtypes = [C.POINTER(ssd_config), C.c_int, _VP, C.POINTER(_VP)]
         L.ssd_load_weights.argtypes = [_VP, C.POINTER(ssd_weights)]
+        L.ssd_w8_read.argtypes = [_VP, C.c_int32, C.c_int32, _VP, _VP]
         L.ssd_kv_create.argtypes = [_VP, C.POINTER(_VP)]
         L.ssd_kv_reset.argtypes = [_VP]
         L.ssd_kv_len.argtypes = [_VP, C.POINTER(C.c_int32)]
@@ -118,7 +120,7 @@ class Context:
     def __init__(self, cfg: dict, device: int = 0, stream: int = 0):
         self.cfg = dict(cfg)
         c = ssd_config(cfg["n_layer"], cfg["d_model"], cfg["n_head"], cfg["d_head"], cfg["d_ff"], cfg["vocab"],
-                       cfg["n_ctx"], cfg["max_nodes"], 1 if cfg["dtype"] == "bf16" else 0, float(cfg["ln_eps"]))
+                       cfg["n_ctx"], cfg["max_nodes"], {"fp32": SSD_DTYPE_F32, "bf16": SSD_DTYPE_BF16, "bf16_w8": SSD_DTYPE_BF16_W8}[cfg["dtype"]], float(cfg["ln_eps"]))
         h = _VP()
         rc = lib().ssd_create(C.byref(c), device, _VP(stream), C.byref(h))
         if rc != SSD_OK:
@@ -140,7 +142,7 @@ class Context:
     def load_weights(self, weights: dict):
         """ssd_load_weights.  ``weights``: numpy arrays, float32 for an fp32 model, uint16 bf16 bit
         patterns for a bf16 model; per-layer entries are lists of n_layer arrays."""
-        want = np.uint16 if self.cfg["dtype"] == "bf16" else np.float32
+        want = np.float32 if self.cfg["dtype"] == "fp32" else np.uint16
         keep, w = [], ssd_weights()
         for k in ("wte", "wpe", "lnf_g", "lnf_b"):
             a = np.ascontiguousarray(weights[k])
@@ -155,6 +157,14 @@ class Context:
             keep.append(tab)
             setattr(w, k, C.cast(tab, _VPP))
         self._chk(lib().ssd_load_weights(self.h, C.byref(w)))
+
+    def w8_read(self, which: int, layer: int = 0):
+        """ssd_w8_read: (codes uint8 [rows, cols], scales float32 [rows]) of one 8-bit matrix (which: 0 w_qkv, 1 w_o, 2 w_fc, 3 w_proj, 4 head)."""
+        d, F, V = self.cfg["d_model"], self.cfg["d_ff"], self.cfg["vocab"]
+        rows, cols = [(3 * d, d), (d, d), (F, d), (d, F), (V, d)][which]
+        codes, scales = np.empty((rows, cols), dtype=np.uint8), np.empty(rows, dtype=np.float32)
+        self._chk(lib().ssd_w8_read(self.h, which, layer, codes.ctypes.data, scales.ctypes.data))
+        return codes, scales
 
     def new_kv(self) -> "KV":
         return KV(self)

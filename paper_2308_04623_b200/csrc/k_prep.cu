@@ -192,3 +192,46 @@ cudaError_t launch_gelu_prep(const float *acc, int n, int F, __nv_bfloat16 *h_hi
     if (grid > 148 * 4) grid = 148 * 4;
     return launch_pdl(gelu_prep_kernel, dim3(grid), dim3(256), s, pdl, acc, count, h_hi, h_lo, trace);
 }
+
+// ---- 8-bit weights: per-row power-of-two scale and e4m3 codes (run once, when the model is loaded) ----
+#include <cuda_fp8.h>
+namespace {
+__global__ void __launch_bounds__(256) quantise_rows_e4m3_kernel(const __nv_bfloat16 *__restrict__ w, size_t cols, uint8_t *__restrict__ codes,
+                                                                 float *__restrict__ scales) {
+    const size_t row = blockIdx.x;
+    const __nv_bfloat16 *src = w + row * cols;
+    __shared__ float part[8];
+    __shared__ float scale_sh;
+    float amax = 0.f;
+    for (size_t k = threadIdx.x; k < cols; k += blockDim.x) amax = fmaxf(amax, fabsf(__bfloat162float(src[k])));
+    for (int o = 16; o; o >>= 1) amax = fmaxf(amax, __shfl_xor_sync(0xffffffffu, amax, o));
+    if ((threadIdx.x & 31) == 0) part[threadIdx.x >> 5] = amax;
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        for (int i = 1; i < 8; ++i) amax = fmaxf(amax, part[i]);
+        // amax = f * 2^x with f in [0.5, 1); 448 = 0.875 * 2^9: the smallest e with amax <= 448 * 2^e
+        float sc = 1.f;
+        if (amax > 0.f && isfinite(amax)) {
+            int x;
+            const float f = frexpf(amax, &x);
+            int e = (f <= 0.875f) ? x - 9 : x - 8;
+            e = e < -100 ? -100 : (e > 100 ? 100 : e);
+            sc = ldexpf(1.f, e);
+        }
+        scale_sh = sc;
+        scales[row] = sc;
+    }
+    __syncthreads();
+    const float inv = 1.f / scale_sh; // (a power of two: exact)
+    for (size_t k = threadIdx.x; k < cols; k += blockDim.x)
+        codes[((row >> 7) * (cols >> 6) + (k >> 6)) * 8192 + (row & 127) * 64 + (k & 63)] =
+            (uint8_t)__nv_cvt_float_to_fp8(__bfloat162float(src[k]) * inv, __NV_SATFINITE, __NV_E4M3);
+}
+} // namespace
+
+size_t w8_tiled_bytes(size_t rows, size_t cols) { return ((rows + 127) / 128) * (cols / 64) * 8192; }
+
+cudaError_t launch_quantise_rows_e4m3(const void *w_bf16, size_t rows, size_t cols, uint8_t *codes, float *scales, cudaStream_t s) {
+    quantise_rows_e4m3_kernel<<<(unsigned)rows, 256, 0, s>>>((const __nv_bfloat16 *)w_bf16, cols, codes, scales);
+    return cudaGetLastError();
+}

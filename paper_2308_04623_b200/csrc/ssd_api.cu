@@ -42,6 +42,9 @@ struct ssd_ctx {
     TensorMap map_wte;
     std::vector<TensorMap> map_layers; // 4 per layer: qkv, o, fc, proj
     bool tensor_path;                  // bf16 model: projections on tcgen05
+    bool w8;                           // bf16 model whose five matrix families are held as e4m3 codes + per-row scales
+    uint8_t *wte8;                     // w8: the output head's codes [vocab, d_model] (the embedding look-up keeps the bf16 table)
+    float *wte_scale;
     int use_lo, pdl, gemm_grid, head_grid, trace_kernels, trace_count, use_graph, use_cluster, cl_max, cl_size[4], attn_lo;
     // cluster-reduced path: per-layer vectors that fold a LayerNorm into the projection behind it (c1 = W gain,
     // c2 = W beta + bias), and the two row-statistics buffers [tile][SSD_MAX_NODES][2] (in front of QKV / of FC)
@@ -184,7 +187,8 @@ static int gemm_grid_for(const ssd_ctx *ctx, int n) {
     if (ctx->gemm_grid > 0) return ctx->gemm_grid;
     return ((n + 15) & ~15) <= 64 ? 2 * ctx->sm_count : ctx->sm_count;
 }
-static int head_grid_for(const ssd_ctx *ctx, int n) { return ctx->head_grid > 0 ? ctx->head_grid : gemm_grid_for(ctx, n); }
+// (8-bit weights: one CTA per SM, whose landing ring is then deep enough to keep the HBM stream of the head busy)
+static int head_grid_for(const ssd_ctx *ctx, int n) { return ctx->head_grid > 0 ? ctx->head_grid : ctx->w8 ? ctx->sm_count : gemm_grid_for(ctx, n); }
 
 // Timeline slots of the next launch (profiling aid, off by default).
 static unsigned long long *trace_slot(ssd_ctx *ctx, int kernels) {
@@ -208,7 +212,7 @@ cudaError_t enqueue_forward(ssd_ctx *ctx, int n, int cap, const NodeList &tk, co
     const GemmHeadStats head_stats = {ctx->head_val, ctx->head_arg, ctx->head_bad};
     const GemmHeadStats *head = (ctx->tensor_path && ctx->use_head_stats) ? &head_stats : nullptr;
     if (ctx->tensor_path && !head) Q(launch_zero_logits(info, n, c.vocab, s));
-    if (ctx->tensor_path && ctx->use_cluster && gemm_cl_supports(n, c.d_model)) {
+    if (ctx->tensor_path && ctx->use_cluster && !ctx->w8 && gemm_cl_supports(n, c.d_model)) {
         // bf16 model, trees of up to 64 nodes: five launches per layer.  Every projection reduces its split-K partial sums
         // inside a thread-block cluster, so its epilogue holds finished sums and does the work that would otherwise be
         // kernels of their own: the LayerNorms are folded (the projection runs on x * gain; mean, rstd and the precomputed
@@ -263,21 +267,22 @@ cudaError_t enqueue_forward(ssd_ctx *ctx, int n, int cap, const NodeList &tk, co
         // accumulate their stream-K partial sums into fp32 buffers; every kernel is a programmatic dependent launch.
         const bool pdl = ctx->pdl != 0;
         const int lo = ctx->use_lo, grid = gemm_grid_for(ctx, n), hgrid = head_grid_for(ctx, n), sms = ctx->sm_count;
+        const bool w8 = ctx->w8;
         __nv_bfloat16 *a_lo = lo ? ctx->a_lo : nullptr, *o_lo = lo ? ctx->o_lo : nullptr, *h_lo = lo ? ctx->h_lo : nullptr;
         for (int l = 0; l < c.n_layer; ++l) {
             const LayerWeights &L = ctx->layers[l];
             const TensorMap *t = &ctx->map_layers[(size_t)4 * l];
             Q(launch_ln_prep(ctx->x, L.ln1_g, L.ln1_b, n, d, c.ln_eps, ctx->a_hi, a_lo, ctx->qkv, 3 * d, info, 0, pdl, s, trace_slot(ctx, *kernels)));
-            Q(launch_gemm_ws(&t[0], &am->a_hi, &am->a_lo, ctx->qkv, info, 3 * d, L.b_qkv, n, d, 3 * d, lo, grid, sms, ctx->d_status, pdl, s, trace_slot(ctx, *kernels)));
+            Q(launch_gemm_ws(&t[0], &am->a_hi, &am->a_lo, ctx->qkv, info, 3 * d, L.b_qkv, n, d, 3 * d, lo, grid, sms, ctx->d_status, pdl, s, trace_slot(ctx, *kernels), nullptr, L.s_qkv, w8 ? (const uint8_t *)L.w_qkv : nullptr));
             Q(launch_tree_attention_mma(ctx->qkv, info, l * layer_elems, ctx->meta, n, c.n_head, cap, ctx->o_hi, o_lo, pdl, s, trace_slot(ctx, *kernels), ctx->attn_lo != 0));
-            Q(launch_gemm_ws(&t[1], &am->o_hi, &am->o_lo, ctx->x, info, d, L.b_o, n, d, d, lo, grid, sms, ctx->d_status, pdl, s, trace_slot(ctx, *kernels)));
+            Q(launch_gemm_ws(&t[1], &am->o_hi, &am->o_lo, ctx->x, info, d, L.b_o, n, d, d, lo, grid, sms, ctx->d_status, pdl, s, trace_slot(ctx, *kernels), nullptr, L.s_o, w8 ? (const uint8_t *)L.w_o : nullptr));
             Q(launch_ln_prep(ctx->x, L.ln2_g, L.ln2_b, n, d, c.ln_eps, ctx->a_hi, a_lo, ctx->h, F, info, 0, pdl, s, trace_slot(ctx, *kernels)));
-            Q(launch_gemm_ws(&t[2], &am->a_hi, &am->a_lo, ctx->h, info, F, L.b_fc, n, d, F, lo, grid, sms, ctx->d_status, pdl, s, trace_slot(ctx, *kernels)));
+            Q(launch_gemm_ws(&t[2], &am->a_hi, &am->a_lo, ctx->h, info, F, L.b_fc, n, d, F, lo, grid, sms, ctx->d_status, pdl, s, trace_slot(ctx, *kernels), nullptr, L.s_fc, w8 ? (const uint8_t *)L.w_fc : nullptr));
             Q(launch_gelu_prep(ctx->h, n, F, ctx->h_hi, h_lo, pdl, s, trace_slot(ctx, *kernels)));
-            Q(launch_gemm_ws(&t[3], &am->h_hi, &am->h_lo, ctx->x, info, d, L.b_proj, n, F, d, lo, grid, sms, ctx->d_status, pdl, s, trace_slot(ctx, *kernels)));
+            Q(launch_gemm_ws(&t[3], &am->h_hi, &am->h_lo, ctx->x, info, d, L.b_proj, n, F, d, lo, grid, sms, ctx->d_status, pdl, s, trace_slot(ctx, *kernels), nullptr, L.s_proj, w8 ? (const uint8_t *)L.w_proj : nullptr));
         }
         Q(launch_ln_prep(ctx->x, ctx->lnf_g, ctx->lnf_b, n, d, c.ln_eps, ctx->a_hi, a_lo, nullptr, 0, info, 0, pdl, s, trace_slot(ctx, *kernels)));
-        Q(launch_gemm_ws(&ctx->map_wte, &am->a_hi, &am->a_lo, nullptr, info, c.vocab, nullptr, n, d, c.vocab, lo, hgrid, sms, ctx->d_status, pdl, s, trace_slot(ctx, *kernels), head));
+        Q(launch_gemm_ws(&ctx->map_wte, &am->a_hi, &am->a_lo, nullptr, info, c.vocab, nullptr, n, d, c.vocab, lo, hgrid, sms, ctx->d_status, pdl, s, trace_slot(ctx, *kernels), head, ctx->wte_scale, ctx->wte8));
         ctx->trace_count = ctx->trace_kernels ? 8 * *kernels : 0;
     } else {
         for (int l = 0; l < c.n_layer; ++l) {
@@ -373,7 +378,7 @@ int ssd_create(const ssd_config *cfg, int device, void *cuda_stream, ssd_ctx **o
     if (out) *out = nullptr;
     if (!cfg || !out) return SSD_ERR_BAD_ARG;
     if (cfg->n_layer < 1 || cfg->d_model < 1 || cfg->n_head < 1 || cfg->d_ff < 1 || cfg->vocab < 1 || cfg->n_ctx < 2 ||
-        cfg->max_nodes < 1 || !(cfg->ln_eps > 0.f) || (cfg->dtype != SSD_DTYPE_F32 && cfg->dtype != SSD_DTYPE_BF16))
+        cfg->max_nodes < 1 || !(cfg->ln_eps > 0.f) || (cfg->dtype != SSD_DTYPE_F32 && cfg->dtype != SSD_DTYPE_BF16 && cfg->dtype != SSD_DTYPE_BF16_W8))
         return SSD_ERR_BAD_ARG;
     if (cfg->d_head != 64 || cfg->n_head * cfg->d_head != cfg->d_model || cfg->d_model % 64 || cfg->d_ff % 64 ||
         cfg->max_nodes > SSD_MAX_NODES || cfg->d_model > 8192)
@@ -383,6 +388,11 @@ int ssd_create(const ssd_config *cfg, int device, void *cuda_stream, ssd_ctx **o
     ssd_ctx *ctx = new (std::nothrow) ssd_ctx();
     if (!ctx) return SSD_ERR_NOMEM;
     ctx->cfg = *cfg;
+    // 8-bit weights change how the matrices are stored and streamed, nothing else: the cache, the activations and every
+    // other kernel are those of the bf16 model
+    ctx->w8 = cfg->dtype == SSD_DTYPE_BF16_W8;
+    if (ctx->w8) ctx->cfg.dtype = SSD_DTYPE_BF16;
+    ctx->wte8 = nullptr; ctx->wte_scale = nullptr;
     ctx->device = device;
     ctx->stream = (cudaStream_t)cuda_stream;
     ctx->loaded = false;
@@ -390,6 +400,7 @@ int ssd_create(const ssd_config *cfg, int device, void *cuda_stream, ssd_ctx **o
     ctx->last_cuda_line = 0;
     ctx->launches = 0;
     ctx->elt = cfg->dtype == SSD_DTYPE_F32 ? 4 : 2;
+    cfg = &ctx->cfg; // (dtype normalised)
     ctx->h_result = nullptr;
     ctx->h_propose = nullptr;
     ctx->d_sparse_idx = nullptr; ctx->d_sparse_val = nullptr; ctx->d_sparse_rows = nullptr;
@@ -516,10 +527,44 @@ int ssd_load_weights(ssd_ctx *ctx, const ssd_weights *w) {
     }
 #undef UP_M
 #undef UP_V
+    if (ctx->w8) {
+        // Quantise on the device: codes and scales in new buffers; a layer's bf16 matrices are released once quantised
+        // (the embedding table stays: the look-up reads it).
+        int rc3;
+        auto quantise = [&](const void *src, size_t rows, size_t cols, const void **codes_out, const float **scales_out) -> int {
+            uint8_t *q = nullptr;
+            float *sc = nullptr;
+            int r = dev_alloc(ctx, &q, w8_tiled_bytes(rows, cols));
+            if (r == SSD_OK) r = dev_alloc(ctx, &sc, rows);
+            if (r != SSD_OK) return r;
+            CU(cudaMemsetAsync(q, 0, w8_tiled_bytes(rows, cols), ctx->stream));
+            CU(launch_quantise_rows_e4m3(src, rows, cols, q, sc, ctx->stream));
+            *codes_out = q; *scales_out = sc;
+            return SSD_OK;
+        };
+        auto release = [&](const void *p) {
+            for (size_t i = ctx->owned.size(); i-- > 0;)
+                if (ctx->owned[i] == p) { ctx->owned.erase(ctx->owned.begin() + (long)i); break; }
+            cudaFree(const_cast<void *>(p));
+        };
+        const void *q8 = nullptr;
+        const float *s8 = nullptr;
+        if ((rc3 = quantise(ctx->wte, c.vocab, d, &q8, &s8)) != SSD_OK) return rc3;
+        ctx->wte8 = (uint8_t *)q8; ctx->wte_scale = (float *)s8;
+        for (int l = 0; l < c.n_layer; ++l) {
+            LayerWeights &L = ctx->layers[l];
+            const void *bf[4] = {L.w_qkv, L.w_o, L.w_fc, L.w_proj};
+            if ((rc3 = quantise(bf[0], 3 * d, d, &L.w_qkv, &L.s_qkv)) != SSD_OK || (rc3 = quantise(bf[1], d, d, &L.w_o, &L.s_o)) != SSD_OK ||
+                (rc3 = quantise(bf[2], F, d, &L.w_fc, &L.s_fc)) != SSD_OK || (rc3 = quantise(bf[3], d, F, &L.w_proj, &L.s_proj)) != SSD_OK)
+                return rc3;
+            CU(cudaStreamSynchronize(ctx->stream));
+            for (const void *p : bf) release(p);
+        }
+    }
     if (ctx->tensor_path) {
         ctx->map_layers.assign((size_t)4 * c.n_layer, TensorMap());
-        int m = make_tensor_map_bf16(&ctx->map_wte, ctx->wte, c.vocab, d, 128);
-        for (int l = 0; l < c.n_layer && m == SSD_OK; ++l) {
+        int m = ctx->w8 ? SSD_OK : make_tensor_map_bf16(&ctx->map_wte, ctx->wte, c.vocab, d, 128);
+        for (int l = 0; l < c.n_layer && m == SSD_OK && !ctx->w8; ++l) { // (8-bit codes are fetched as contiguous tiles: no maps)
             const LayerWeights &L = ctx->layers[l];
             TensorMap *t = &ctx->map_layers[(size_t)4 * l];
             m = make_tensor_map_bf16(&t[0], L.w_qkv, 3 * d, d, 128);
@@ -531,7 +576,7 @@ int ssd_load_weights(ssd_ctx *ctx, const ssd_weights *w) {
         // LayerNorm-fold vectors of the cluster-reduced path, its statistics buffers, the timeline buffer
         int rc2;
         ctx->folds.assign(c.n_layer, ssd_ctx::LayerFold());
-        for (int l = 0; l < c.n_layer; ++l) {
+        for (int l = 0; l < c.n_layer && !ctx->w8; ++l) { // (the cluster-reduced path does not take 8-bit weights)
             const LayerWeights &L = ctx->layers[l];
             ssd_ctx::LayerFold &f = ctx->folds[l];
             if ((rc2 = dev_alloc(ctx, &f.c1_qkv, 3 * d)) != SSD_OK || (rc2 = dev_alloc(ctx, &f.c2_qkv, 3 * d)) != SSD_OK ||
@@ -548,6 +593,34 @@ int ssd_load_weights(ssd_ctx *ctx, const ssd_weights *w) {
     }
     CU(cudaStreamSynchronize(ctx->stream));
     ctx->loaded = true;
+    return SSD_OK;
+}
+
+int ssd_w8_read(ssd_ctx *ctx, int32_t which, int32_t layer, uint8_t *codes_out, float *scales_out) {
+    if (!ctx || !codes_out || !scales_out || !ctx->w8 || which < 0 || which > 4) return SSD_ERR_BAD_ARG;
+    if (!ctx->loaded) return SSD_ERR_NOT_LOADED;
+    if (which < 4 && (layer < 0 || layer >= ctx->cfg.n_layer)) return SSD_ERR_BAD_ARG;
+    DeviceGuard g(ctx->device);
+    if (!g.ok) return SSD_ERR_CUDA;
+    const size_t d = ctx->cfg.d_model, F = ctx->cfg.d_ff;
+    const void *codes = ctx->wte8;
+    const float *scales = ctx->wte_scale;
+    size_t rows = ctx->cfg.vocab, cols = d;
+    if (which < 4) {
+        const LayerWeights &L = ctx->layers[layer];
+        const void *cw[4] = {L.w_qkv, L.w_o, L.w_fc, L.w_proj};
+        const float *sw[4] = {L.s_qkv, L.s_o, L.s_fc, L.s_proj};
+        const size_t rw[4] = {3 * d, d, F, d}, kw[4] = {d, d, d, F};
+        codes = cw[which]; scales = sw[which]; rows = rw[which]; cols = kw[which];
+    }
+    std::vector<uint8_t> tiled(w8_tiled_bytes(rows, cols)); // stored tile by tile; handed back row-major
+    CU(cudaMemcpyAsync(tiled.data(), codes, tiled.size(), cudaMemcpyDeviceToHost, ctx->stream));
+    CU(cudaMemcpyAsync(scales_out, scales, rows * sizeof(float), cudaMemcpyDeviceToHost, ctx->stream));
+    CU(cudaStreamSynchronize(ctx->stream));
+    const size_t k_tiles = cols / 64;
+    for (size_t o = 0; o < rows; ++o)
+        for (size_t kt = 0; kt < k_tiles; ++kt)
+            memcpy(codes_out + o * cols + kt * 64, tiled.data() + ((o / 128) * k_tiles + kt) * 8192 + (o % 128) * 64, 64);
     return SSD_OK;
 }
 

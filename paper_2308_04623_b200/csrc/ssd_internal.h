@@ -37,7 +37,8 @@ struct StepInfo {
 
 struct LayerWeights {
     const float *ln1_g, *ln1_b, *b_qkv, *b_o, *ln2_g, *ln2_b, *b_fc, *b_proj; // fp32 on device
-    const void *w_qkv, *w_o, *w_fc, *w_proj;                                  // float or bf16
+    const void *w_qkv, *w_o, *w_fc, *w_proj;                                  // float or bf16; e4m3 codes when the weights are 8-bit
+    const float *s_qkv, *s_o, *s_fc, *s_proj;                                 // 8-bit weights: one scale per output row
 };
 
 enum GemmEpilogue { EPI_STORE = 0, EPI_GELU = 1, EPI_RESIDUAL = 2 };
@@ -72,6 +73,12 @@ cudaError_t launch_gelu_prep(const float *acc, int n, int F, __nv_bfloat16 *h_hi
 // Tensor maps are opaque 128-byte objects (CUtensorMap) built on the host.
 struct alignas(64) TensorMap { unsigned char bytes[128]; };
 int make_tensor_map_bf16(void *map_out, const void *base, uint64_t rows, uint64_t cols, uint32_t box_rows);
+// 8-bit weights: W[rows, cols] bf16 -> e4m3 codes and one power-of-two scale per row, the smallest that brings the row's
+// largest magnitude within the format's range (448); code = round-to-nearest-even(W / scale).  A row of zeros gets scale 1.
+// The codes are written tile by tile: code (o, k) at ((o / 128) * (cols / 64) + k / 64) * 8192 + (o % 128) * 64 + k % 64; the
+// buffer holds ceil(rows / 128) * (cols / 64) tiles and must be zeroed beforehand (rows past the matrix stay zero).
+size_t w8_tiled_bytes(size_t rows, size_t cols);
+cudaError_t launch_quantise_rows_e4m3(const void *w_bf16, size_t rows, size_t cols, uint8_t *codes, float *scales, cudaStream_t s);
 cudaError_t gemm_ws_prepare();
 cudaError_t prep_kernels_prepare();
 // y[n, ldy] += X[n, K] . W[out, K]^T (+ bias once).  map_w: weights [out, K], boxes of 128 rows; map_hi / map_lo:
@@ -80,10 +87,13 @@ cudaError_t prep_kernels_prepare();
 // half an SM's shared memory.
 // With `head` set the projection runs one CTA per output tile over the whole K (complete sums): plain stores, no clearing of Y
 // needed, and per (row, tile) the maximum, its lowest feature index and a non-finite flag at [row * n_tiles + tile].
+// With `w_codes` set the weights are 8-bit codes stored tile by tile (see launch_quantise_rows_e4m3), w_scale[out] their per-row
+// scales, and map_w is ignored.
 struct GemmHeadStats { float *val; int32_t *arg, *bad; };
 cudaError_t launch_gemm_ws(const void *map_w, const void *map_hi, const void *map_lo, float *y, const StepInfo *info, int ldy,
                            const float *bias, int n, int K, int out, int use_lo, int grid, int sm_count, int32_t *status, bool pdl,
-                           cudaStream_t s, unsigned long long *trace = nullptr, const GemmHeadStats *head = nullptr);
+                           cudaStream_t s, unsigned long long *trace = nullptr, const GemmHeadStats *head = nullptr,
+                           const float *w_scale = nullptr, const uint8_t *w_codes = nullptr);
 // ---- projection with the split-K sums reduced inside a thread-block cluster (trees of up to 64 nodes) ----
 // What the epilogue does with the finished sums acc[i, o] (see k_gemm_cl.cu):
 enum { MODE_FOLD_STORE = 0, MODE_FOLD_GELU = 1, MODE_RESIDUAL = 2 };

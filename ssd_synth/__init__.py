@@ -90,7 +90,7 @@ def make_weights(cfg: dict, seed: int = 0, qk_gain: float = 1.0) -> dict:
     """
     rng = np.random.default_rng(seed)
     L, d, F, V, C = cfg["n_layer"], cfg["d_model"], cfg["d_ff"], cfg["vocab"], cfg["n_ctx"]
-    bf16 = cfg["dtype"] == "bf16"
+    bf16 = cfg["dtype"] != "fp32"   # ("bf16_w8": a bf16 model whose matrices the library holds as 8-bit codes)
 
     def normal(*shape):
         return (rng.standard_normal(shape, dtype=np.float32) * np.float32(0.02))
@@ -261,8 +261,11 @@ def trigram_tree(prev2: int, prev1: int, root_token: int, vocab: int, seed: int 
 # ----------------------------------------------------------------------------
 def algorithmic_bytes(cfg: dict, prefix: int, n_nodes: int) -> int:
     L, d, F, V = cfg["n_layer"], cfg["d_model"], cfg["d_ff"], cfg["vocab"]
-    wb = 2 if cfg["dtype"] == "bf16" else 4
-    weights = wb * (L * (4 * d * d + 2 * d * F + 9 * d + F) + V * d)
+    wb = 4 if cfg["dtype"] == "fp32" else 2
+    mb = 1 if cfg["dtype"] == "bf16_w8" else wb          # bytes per matrix entry
+    matrices = L * (4 * d * d + 2 * d * F) + V * d
+    scales = 4 * (L * (5 * d + F) + V) if cfg["dtype"] == "bf16_w8" else 0   # one fp32 scale per output row
+    weights = mb * matrices + scales + wb * L * (9 * d + F)
     kv = L * 2 * d * wb * (prefix + 2 * n_nodes)
     logits = 4 * n_nodes * V
     return weights + kv + logits

@@ -4,19 +4,22 @@ import torch
 
 import ssd_synth
 import paper_2308_04623_b200 as ssd
-from oracle import ssd_oracle
+from oracle import ssd_oracle, w8_oracle
 
 
 class Pair:
     """One model held by the CUDA library and by the oracle, each with its own cache."""
 
-    def __init__(self, cfg_name, seed=0, qk_gain=1.0, **overrides):
+    def __init__(self, cfg_name, seed=0, qk_gain=1.0, on_grid=False, **overrides):
         self.cfg = ssd_synth.config(cfg_name, **overrides)
         w = ssd_synth.make_weights(self.cfg, seed=seed, qk_gain=qk_gain)
+        if on_grid:  # the streamed matrices moved onto the 8-bit code grid: the 8-bit library model and the oracle hold the same numbers
+            w = w8_oracle.model_on_the_grid(w)
+        self.weights = w
         self.oracle = ssd_oracle.Model(self.cfg, w)
         self.okv = self.oracle.new_kv()
         self.ctx = ssd.Context(self.cfg, device=0, stream=torch.cuda.current_stream().cuda_stream)
-        self.ctx.load_weights(ssd_synth.bf16_bits(w) if self.cfg["dtype"] == "bf16" else w)
+        self.ctx.load_weights(ssd_synth.bf16_bits(w) if self.cfg["dtype"] != "fp32" else w)
         self.kv = self.ctx.new_kv()
         self.V = self.cfg["vocab"]
 

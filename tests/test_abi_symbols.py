@@ -14,7 +14,7 @@ def test_library_builds_loads_and_exports_all_declared_symbols():
     import paper_2308_04623_b200 as ssd
     lib = ssd.lib()
     header = open(os.path.join(ROOT, "include", "ssd.h")).read()
-    declared = set(re.findall(r"\b(ssd_[a-z_]+)\s*\(", header))
+    declared = set(re.findall(r"\b(ssd_[a-z0-9_]+)\s*\(", header))
     assert declared, "no declarations found"
     assert declared == set(ssd.EXPORTS)
     for name in declared:

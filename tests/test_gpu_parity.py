@@ -719,3 +719,85 @@ def test_proposed_children_follow_the_nodes_laws(ssd):
         assert e.value.code == ssd.SSD_ERR_BAD_ARG
     finally:
         ctx.close()
+
+
+# ---------------------------------------------------------------------------
+# 8-bit weight streaming (Section 4, closing list of next steps)
+# ---------------------------------------------------------------------------
+def test_w8_device_encoding_matches_the_oracle_encoding(ssd):
+    """Arbitrary bf16 matrices: the codes and scales the library holds are, bit for bit, those of the encoding's definition."""
+    from oracle import w8_oracle
+    cfg = ssd_synth.config("ragged_bf16", dtype="bf16_w8")
+    w = ssd_synth.make_weights(cfg, seed=21)
+    w["w_fc"][1][5, :] = 0.0                     # a row of zeros
+    w["w_o"][0][7, 3] = ssd_synth.round_to_bf16(np.float32([3.7]))[0]   # a row with one dominant entry: the others fall into the sub-normal codes
+    ctx = ssd.Context(cfg, device=0, stream=torch.cuda.current_stream().cuda_stream)
+    ctx.load_weights(ssd_synth.bf16_bits(w))
+    for which, name in enumerate(w8_oracle.MATRICES):
+        for l in range(cfg["n_layer"]):
+            codes, scales = ctx.w8_read(which, l)
+            want_c, want_s = w8_oracle.quantise_rows(w[name][l])
+            assert np.array_equal(scales, want_s), (name, l)
+            assert np.array_equal(codes & 0x7F, want_c & 0x7F) and np.array_equal((codes >> 7)[(codes & 0x7F) != 0], (want_c >> 7)[(want_c & 0x7F) != 0]), (name, l)
+    codes, scales = ctx.w8_read(4)
+    want_c, want_s = w8_oracle.quantise_rows(w["wte"])
+    assert np.array_equal(scales, want_s) and np.array_equal(codes & 0x7F, want_c & 0x7F)
+    sub = (codes & 0x7F) < 8
+    assert sub.any()                              # sub-normal codes occur in these matrices
+    # another dtype has nothing to read
+    with pytest.raises(ssd.SsdError):
+        ssd.Context(ssd_synth.config("ragged_bf16")).w8_read(0, 0)
+    ctx.close()
+
+
+@pytest.mark.parametrize("cfg_name", ["ragged_bf16", "tiny_bf16"])
+def test_w8_logits_against_the_oracle_and_the_bf16_path(ssd, util, cfg_name):
+    """The model on the code grid held three ways - by the oracle (fp64), by the library as bf16 and by the library as 8-bit
+    codes: 8-bit against the oracle within the bf16 tolerance over trees that span the single- and two-instruction operand
+    layouts and ragged tails, with commits in between; 8-bit against bf16 to summation-order noise (same numbers, same
+    products; only the order of the fp32 additions differs); same number of launches."""
+    rng = np.random.default_rng(31)
+    p8 = util.Pair(cfg_name, seed=4, on_grid=True, dtype="bf16_w8")
+    p16 = util.Pair(cfg_name, seed=4, on_grid=True)
+    V = p8.V
+    prefix = ssd_synth.uniform_tokens(70, V, rng)
+    p8.prefill(prefix); p16.prefill(prefix)
+    L = p8.cfg["n_layer"]
+    for n in (1, 5, 29, 64, 100, 256):
+        par = ssd_synth.tree_random(n, 8, rng)
+        tok = ssd_synth.uniform_tokens(n, V, rng)
+        before = p8.ctx.kernel_launches()
+        got8, want, buf8 = p8.verify(tok, par)
+        assert p8.ctx.kernel_launches() - before == 3 + 8 * L + 2
+        got16, _, _ = p16.verify(tok, par)
+        assert np.isfinite(got8).all()
+        assert np.abs(got8 - want).max() <= TOL_BF16, n
+        assert np.abs(got8 - got16).max() <= 1e-3, n
+        path, nxt = p8.ctx.accept_tree(buf8.data_ptr(), None, tok, par)
+        opath, onext, margin = ssd_oracle.accept_tree(want.astype(np.float32), None, tok, par)
+        if margin > 4 * TOL_BF16:
+            assert list(path) == list(opath) and nxt == onext
+        p8.commit(opath[:3]); p16.commit(opath[:3])
+    assert p8.ctx.device_status() == 0
+    p8.close(); p16.close()
+
+
+@pytest.mark.parametrize("ctas", [1, 2, 5])
+def test_w8_with_few_ctas_streams_through_the_landing_ring(ssd, util, ctas):
+    """With few CTAs each one holds more units than stages, so the 8-bit tiles go through the ring of landing slots and the
+    dedicated converter warps (at full size only the LM head does): same logits as the oracle, for the layer projections and
+    the head alike, over several steps (the barriers' phases wrap more than once)."""
+    rng = np.random.default_rng(41 + ctas)
+    p8 = util.Pair("ragged_bf16", seed=6, on_grid=True, dtype="bf16_w8")
+    p8.ctx.set_tuning(ssd.SSD_TUNE_GEMM_CTAS, ctas)
+    p8.ctx.set_tuning(ssd.SSD_TUNE_HEAD_CTAS, ctas)
+    V = p8.V
+    p8.prefill(ssd_synth.uniform_tokens(37, V, rng))
+    for n in (3, 40, 130):
+        par = ssd_synth.tree_random(n, 6, rng)
+        tok = ssd_synth.uniform_tokens(n, V, rng)
+        got8, want, _ = p8.verify(tok, par)
+        assert np.abs(got8 - want).max() <= TOL_BF16, (ctas, n)
+        p8.commit([0])
+    assert p8.ctx.device_status() == 0
+    p8.close()

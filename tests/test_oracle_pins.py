@@ -231,3 +231,69 @@ def test_greedy_tree_decoding_equals_autoregressive(tiny_model):
         steps += 1
     assert got[:n_new] == want
     assert steps < n_new  # speculation did accept something
+
+
+# ---------------------------------------------------------------------------
+# 8-bit weight encoding (e4m3 codes + per-row power-of-two scale)
+# ---------------------------------------------------------------------------
+def test_e4m3_table_landmarks():
+    """The code table against the format's published landmarks: 0x38 = 1, 0x7e = 448 (largest), 0x08 = 2^-6 (smallest
+    normal), 0x01 = 2^-9 (smallest sub-normal), 0x7f not a number, 126 positive values strictly ascending, sign symmetric."""
+    from oracle import w8_oracle
+    v = w8_oracle.code_values()
+    assert v[0x00] == 0.0 and v[0x38] == 1.0 and v[0x7E] == 448.0 and v[0x08] == 2.0 ** -6 and v[0x01] == 2.0 ** -9
+    assert v[0x40] == 2.0 and v[0x3C] == 1.5 and v[0x07] == 7 * 2.0 ** -9
+    assert np.isnan(v[0x7F]) and np.isnan(v[0xFF])
+    assert np.all(np.diff(v[:127]) > 0)
+    assert np.array_equal(v[128:255], -v[0:127])
+
+
+def test_e4m3_encode_ties_saturation_and_grid():
+    from oracle import w8_oracle
+    enc, v = w8_oracle.encode, w8_oracle.code_values()
+    # ties go to the even pattern: 1.0625 lies between 1.0 (0x38) and 1.125 (0x39); 1.1875 between 0x39 and 1.25 (0x3a)
+    assert list(enc([1.0625, 1.1875, -1.0625, -1.1875])) == [0x38, 0x3A, 0xB8, 0xBA]
+    # across an exponent boundary: 1.9375 is halfway between 1.875 (0x3f) and 2.0 (0x40)
+    assert list(enc([1.9375])) == [0x40]
+    # sub-normal ties: 2^-10 is halfway between 0 and 2^-9 -> 0; 3 * 2^-10 halfway between codes 1 and 2 -> 2
+    assert list(enc([2.0 ** -10, 3 * 2.0 ** -10])) == [0x00, 0x02]
+    assert list(enc([1e9, -1e9, 448.0, 464.0, 0.0])) == [0x7E, 0xFE, 0x7E, 0x7E, 0x00]
+    # every finite code encodes to itself
+    codes = np.array([c for c in range(256) if c not in (0x7F, 0xFF, 0x80)], dtype=np.uint8)
+    assert np.array_equal(enc(v[codes]), codes)
+
+
+def test_e4m3_encode_matches_torch_cast_in_range():
+    """A library routine as the pin: torch's float8_e4m3fn cast rounds to nearest even too (in range; it does not saturate)."""
+    from oracle import w8_oracle
+    rng = np.random.default_rng(5)
+    x = np.concatenate([rng.standard_normal(20000) * s for s in (1e-3, 0.05, 1.0, 30.0, 150.0)]).astype(np.float32)
+    x = x[np.abs(x) <= 448.0]
+    want = torch.from_numpy(x).to(torch.float8_e4m3fn).view(torch.uint8).numpy()
+    got = w8_oracle.encode(x.astype(np.float64))
+    same = (got == want) | ((x == 0) & ((got & 0x7F) == 0) & ((want & 0x7F) == 0))
+    assert same.all()
+
+
+def test_w8_row_scale_rule_and_error_bound():
+    from oracle import w8_oracle
+    w = np.zeros((6, 8), dtype=np.float32)
+    w[0, 3] = 448.0; w[1, 0] = -449.0; w[2, 7] = 224.0; w[3, 1] = 224.5; w[5, 2] = 0.02
+    s = w8_oracle.row_scales(w)
+    assert list(s[:5]) == [1.0, 2.0, 0.5, 1.0, 1.0]           # (row 4 is all zeros)
+    assert s[5] == 2.0 ** -14 and 0.02 <= 448 * s[5] and 0.02 > 448 * s[5] / 2
+    # decode(encode(w)) differs from w by at most half a code step: relative 2^-4 in the normal range, absolute
+    # scale * 2^-10 below it
+    rng = np.random.default_rng(11)
+    W = (rng.standard_normal((64, 512)) * 0.02).astype(np.float32)
+    q, sc = w8_oracle.quantise_rows(W)
+    D = w8_oracle.dequantise_rows(q, sc)
+    err = np.abs(D.astype(np.float64) - W)
+    bound = np.maximum(np.abs(W) * 2.0 ** -4, sc[:, None].astype(np.float64) * 2.0 ** -10)
+    assert (err <= bound).all()
+    assert (np.abs(q.astype(np.int32) & 0x7F).max(axis=1) >= 0x70).all()   # every row uses the top octave of the format
+    # on its own grid the encoding is lossless, whatever scale the second pass picks
+    q2, sc2 = w8_oracle.quantise_rows(D)
+    assert np.array_equal(w8_oracle.dequantise_rows(q2, sc2), D)
+    # and the grid values are bf16 numbers
+    assert np.array_equal(ssd_synth.round_to_bf16(D), D)
