@@ -420,6 +420,27 @@ def run_sweep(args, local, peaks):
     return out
 
 
+def run_w8(args, local, peaks):
+    """8-bit weight streaming (the paper's closing list of next steps, item 2) beside the bf16 model, same trees and tokens: verify time, the
+    algorithmic bytes of each (codes of one byte and a scale per row against two bytes) and the fraction of the copy bandwidth."""
+    out = []
+    steps = max(10, min(args.steps, 30))
+    for model, P, n in ((args.model, args.prefix, 32), ("gpt2_xl", 512, 32)):
+        par = ssd_synth.tree_branching(n, tree_rule(n))
+        row = {"workload": "%s verify n=%d prefix=%d" % (model, n, P)}
+        for dtype in ("bf16", "bf16_w8"):
+            run = Runner(model, P, local, args.tune, dtype=dtype)
+            toks = [ssd_synth.uniform_tokens(n, run.V, run.rng) for _ in range(4)]
+            e = sweep_entry(model, run.cfg, n, P, run.time_steps(par, toks, steps, 3), peaks)
+            row[dtype] = {k: e[k] for k in ("verify_us", "algorithmic_bytes", "achieved_gbs", "frac_hbm_measured", "bound_us")}
+            run.close()
+            del run
+        row["w8_time_over_bf16"] = row["bf16_w8"]["verify_us"]["median"] / row["bf16"]["verify_us"]["median"]
+        out.append(row)
+    return {"rows": out, "note": "codes go to the 8-bit tensor-core kind unconverted; activations as four e4m3 planes; the forward is a chain of "
+                                 "dependent kernels, so halving the streamed bytes moves the LM head (HBM-bound) and little else"}
+
+
 def run_staged(args, local, peaks, alphas=(0.3, 0.6, 0.9), n_tokens=256):
     """The full staged loop at the benchmark's sizes with the acceptance made controllable: GPT-2-Large-shaped target,
     GPT-2-small-shaped draft, a trigram table built from a synthetic stream.  Random-weight models never agree, so - as
@@ -598,6 +619,7 @@ def run_gpu(args):
             del r2
         sweep.update(run_sweep(args, local, peaks))
         sweep["config4"] = run_staged(args, local, peaks)
+        sweep["w8"] = run_w8(args, local, peaks)
         line["sweep"] = sweep
     if world == 1 and not args.no_cpu_baseline:
         times = oracle_steps(cfg, weights, parent, P, np.random.default_rng(7), 3, 0, 60.0)

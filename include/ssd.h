@@ -60,10 +60,16 @@ typedef struct {
  * given and run as the bf16 model, but ssd_load_weights re-encodes the matrices the projections stream - w_qkv, w_o,
  * w_fc, w_proj and the output head (wte) - as e4m3 codes (1 sign, 4 exponent, 3 fraction bits) with one fp32 scale per
  * output row, halving the bytes a step reads.  The scale of a row is the smallest power of two s with max|w| <= 448 s
- * (1 for a row of zeros); code = round-to-nearest-even(w / s), saturating; the kernels compute with code * s exactly
- * (the codes are widened to bf16 on chip, the scale multiplies the fp32 sums).  A matrix whose entries are already
- * code * power-of-two values is therefore represented without loss.  The embedding look-up keeps the bf16 table;
- * biases, LayerNorm parameters, activations and the cache are as with dtype 1.
+ * (1 for a row of zeros); code = round-to-nearest-even(w / s), saturating; the kernels compute with code * s exactly:
+ * the codes go to the tensor cores as they are (the 8-bit kind of tcgen05.mma, fp32 accumulation) and the scale
+ * multiplies the fp32 sums.  A matrix whose entries are already code * power-of-two values is therefore represented
+ * without loss.  That instruction kind wants its other operand in an 8-bit format too, so the kernels that produce the
+ * projections' inputs write each value as four e4m3 planes, x = 16 p0 + p1 + p2 / 16 + p3 / 256 to about 16
+ * significant bits (what the bf16 model's hi + lo operand pair carries; |x| up to 7168 before the first plane
+ * saturates); SSD_TUNE_W8_PLANES can drop the last ones.  A projection launch takes at most 128 nodes, so a larger
+ * tree runs each projection as two launches.  The embedding look-up keeps the bf16 table; biases, LayerNorm
+ * parameters, the attention and the cache are as with dtype 1.  SSD_TUNE_CLUSTER_REDUCE and SSD_TUNE_HEAD_STATS
+ * have no effect on such a context.
  */
 enum { SSD_DTYPE_F32 = 0, SSD_DTYPE_BF16 = 1, SSD_DTYPE_BF16_W8 = 2 };
 enum { SSD_GREEDY = 0, SSD_SAMPLING = 1 };
@@ -267,11 +273,13 @@ int ssd_kv_read(ssd_ctx *ctx, const ssd_kv *kv, int32_t layer, int32_t which, in
  *                                 context wrote (same n_nodes, buffer not modified in between) reads those instead of the logits.
  *                                 Measured: the forward 10 us slower (393 tiles over 296 CTA slots leave a ragged last wave), the
  *                                 acceptance 10 us faster.  0 = stream-K head adding partial sums at L2 into cleared logits
+ *   SSD_TUNE_W8_PLANES [4]        SSD_DTYPE_BF16_W8 only: how many e4m3 planes of an activation the projections use, 2..4 (each carries
+ *                                 4 significant bits; every plane less shortens the projections' epilogues)
  *   SSD_TUNE_KERNEL_TRACE [0]     record a timeline of every kernel of a bf16 forward (see ssd_get_phase_trace)
  */
 enum { SSD_TUNE_LOW_PLANE = 0, SSD_TUNE_DEPENDENT_LAUNCH = 1, SSD_TUNE_GRAPH = 2, SSD_TUNE_GEMM_CTAS = 3, SSD_TUNE_CLUSTER_REDUCE = 4,
        SSD_TUNE_CLUSTER_MAX = 5, SSD_TUNE_ATTN_LOW_PLANE = 6, SSD_TUNE_HEAD_CTAS = 7, SSD_TUNE_KERNEL_TRACE = 8, SSD_TUNE_CLUSTER_QKV = 9, SSD_TUNE_CLUSTER_O = 10,
-       SSD_TUNE_CLUSTER_FC = 11, SSD_TUNE_CLUSTER_PROJ = 12, SSD_TUNE_HEAD_STATS = 13 };
+       SSD_TUNE_CLUSTER_FC = 11, SSD_TUNE_CLUSTER_PROJ = 12, SSD_TUNE_HEAD_STATS = 13, SSD_TUNE_W8_PLANES = 14 };
 int ssd_set_tuning(ssd_ctx *ctx, int32_t knob, int32_t value);
 
 /*

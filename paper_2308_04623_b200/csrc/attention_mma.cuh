@@ -21,6 +21,7 @@
 #pragma once
 #include "sm100_ptx.cuh"
 #include "ssd_internal.h"
+#include "w8_planes.cuh"
 
 namespace attn {
 constexpr int DH = 64;
@@ -42,6 +43,8 @@ struct Output {
     float *part_o;              // several splits: [split][max_nodes][d] un-normalised sums
     float *part_ml;             // several splits: [split][max_nodes][n_head][2] running max and sum
     int max_nodes, n_head;
+    uint8_t *planes8;           // one split, 8-bit projections: the output as four e4m3 planes [4][rows][d] instead of o_hi / o_lo
+    size_t plane_stride;
 };
 
 __device__ __forceinline__ void mma_bf16(float (&c)[4], const uint32_t (&a)[4], uint32_t b0, uint32_t b1) {
@@ -328,6 +331,7 @@ __device__ __forceinline__ void work_item(int tid, int bar_id, unsigned char *sm
             const size_t at = (size_t)row * d + h * DH + c0;
             if (n_splits == 1) {
                 const float inv = 1.0f / L; // a node always sees itself, so L > 0
+                if (out.planes8) { w8::store4(out.planes8, out.plane_stride, at, acc[0] * inv, acc[1] * inv, acc[2] * inv, acc[3] * inv); continue; }
                 uint32_t h0, l0, h1, l1;
                 split_pair(acc[0] * inv, acc[1] * inv, h0, l0);
                 split_pair(acc[2] * inv, acc[3] * inv, h1, l1);

@@ -26,21 +26,15 @@
 //     hold no integer division and no per-unit fence or commit, and the epilogue fetches what
 //     does not depend on the accumulator before it waits for it;
 //   * every wait is bounded; on a time-out the CTA records an error word and unwinds;
-//   * 8-bit weights (the W8 instantiation; Section 4's closing list names 8-bit quantisation as the next step):
-//     the matrix is stored as e4m3 codes with one fp32 scale per output row, so half the bytes stream from HBM.
-//     The codes are stored tile by tile - the [128 rows x 64 codes] of an (output tile, k tile) unit are 8 KB in a row,
-//     rows past the matrix zero - so a unit arrives as ONE contiguous copy (rows of 64 bytes fetched one by one from a
-//     row-major matrix use a fraction of every DRAM burst and of every 256-byte L2 fetch).
-//     A tile is widened on chip to bf16, in the swizzled layout the tensor cores read (both MMA operands stay bf16).
-//     When a CTA has no more units than stages (the projections of a layer), a tile lands in the upper half of its
-//     stage's own 16 KB weight buffer and the four epilogue warps, which have nothing else to do yet, widen it in place
-//     (through registers, a barrier between the reads and the writes): the CTA has the threads and the shared memory of
-//     the bf16 kernel, so the next kernels' CTAs stay resident beside it.  Otherwise (the LM head) tiles land in a
-//     ring of 8 KB slots behind a short ring of stages - a deep, cheap ring that covers the HBM latency -, eight more
-//     warps widen them, four units at a time (the epilogue warps help with the CTA's first units), and refill a slot
-//     themselves as soon as they have read it.
-//     The epilogue multiplies the sums by the row's scale.  The widening needs no activations, so it too runs ahead
-//     of the dependency wait.
+//   * 8-bit weights (the W8 instantiation; Section 4's closing list names 8-bit quantisation as the next step): the
+//     matrix is stored as e4m3 codes with one fp32 scale per output row, so half the bytes stream from HBM, and it
+//     goes to the tensor cores as it is - the 8-bit kind of tcgen05.mma, 32 codes of K per instruction, a weight
+//     tile of [128 rows x 128 codes] per stage.  No thread touches a weight.  The activations, which that kind wants
+//     in an 8-bit format too, arrive as FOUR e4m3 planes (see w8_planes.cuh: x = 16 p0 + p1 + p2 / 16 + p3 / 256 to
+//     about 16 significant bits, what the bf16 hi + lo pair carries); the planes are stacked along N, so one
+//     instruction multiplies a weight slice by all four (N = 4 n_pad <= 256; two instructions for 128 rows), each
+//     plane's product in accumulator columns of its own.  The epilogue adds the four with their powers of two and
+//     multiplies by the row's scale.  At most 128 rows per launch (512 accumulator columns).
 #include <cuda.h>
 #include <cstring>
 
@@ -53,11 +47,8 @@ constexpr int TILE_K = 64;                  // bf16 elements per k tile = 128 by
 constexpr int UMMA_K = 16;                  // k per tcgen05.mma for 16-bit inputs
 constexpr int A_BYTES = TILE_M * TILE_K * 2;  // 16 KB
 constexpr int MAX_STAGES = 12;
-constexpr int MAX_LANDING = 16;               // W8: landing slots
-constexpr int A8_BYTES = TILE_M * TILE_K;     // 8 KB: the same tile as 8-bit codes
+constexpr int W8_PLANES = 4;                // e4m3 planes an activation is split into
 constexpr int GEMM_THREADS = 192;
-constexpr int W8_PAIRS = 4;                   // pairs of dedicated converter warps (landing-ring mode)
-constexpr int GEMM_THREADS_W8 = GEMM_THREADS + 64 * W8_PAIRS;
 constexpr int SMEM_BUDGET = 210 * 1024;   // stages of one CTA per SM (the barriers and the statistics scratch follow them)
 constexpr int SMEM_BUDGET_SHARED = 106 * 1024;
 #ifndef EPI_POLL_NS
@@ -73,12 +64,12 @@ struct GemmParams {
     int k_tiles;       // K / 64
     int n_tiles;       // ceil(out / 128)
     int stages;
-    int landing;       // W8: landing slots of 8 KB behind the stages; 0 = tiles land inside their stage (units <= stages)
     int split;         // > 0: every output tile's k tiles are shared by `split` CTAs of its own (grid = split * n_tiles); 0: stream-K ranges
     int use_lo;
     int32_t *status;   // device error word
-    const float *w_scale; // [out] scale of each output row's 8-bit codes (W8 only)
-    const uint8_t *w_codes; // W8: [n_tiles][k_tiles][128][64] codes
+    const float *w_scale; // W8: [out] scale of each output row's codes
+    int planes;        // W8: how many of the four e4m3 planes of the activations take part (2..4)
+    int row0;          // first activation row (node) of this launch (W8 with more than 128 nodes runs in two launches)
     // LM head with complete sums (split == 1): plain stores instead of reductions, and per (row, output tile) the maximum,
     // its lowest index and a non-finite flag, so that greedy acceptance need not read the logits again
     int store;
@@ -92,8 +83,6 @@ struct __align__(8) Barriers {
     int32_t stat_arg[4][SSD_MAX_NODES];
     int32_t stat_bad[4];
     uint64_t full[MAX_STAGES];
-    uint64_t wfull[MAX_LANDING];        // W8: a landing slot's 8-bit tile has arrived
-    uint64_t wempty[MAX_LANDING];       // W8: the converters have read it
     uint64_t empty[MAX_STAGES];
     uint64_t acc_full[2];
     uint64_t acc_empty[2];
@@ -109,100 +98,18 @@ __device__ __forceinline__ void fail(const GemmParams &p, Barriers *b, int code)
 }
 
 
-// Four e4m3 codes (one 32-bit word, lowest byte first) as four bf16 values in two words.  A code's seven magnitude bits
-// placed at bits 4..10 of a bf16 give the same number scaled by 2^-120, sub-normal codes included (they become sub-normal
-// bf16 values with the same fraction); one packed multiplication by 2^120 - exact - restores the scale.
-__device__ __forceinline__ void e4m3x4_to_bf16x4(uint32_t w, uint32_t &lo, uint32_t &hi) {
-    const uint32_t x01 = __byte_perm(w, 0u, 0x1404), x23 = __byte_perm(w, 0u, 0x3424); // codes in the high byte of each half
-    const uint32_t b01 = (x01 & 0x80008000u) | ((x01 >> 4) & 0x07f007f0u);
-    const uint32_t b23 = (x23 & 0x80008000u) | ((x23 >> 4) & 0x07f007f0u);
-    const uint32_t two120 = 0x7B807B80u;
-    asm("mul.rn.bf16x2 %0, %1, %2;" : "=r"(lo) : "r"(b01), "r"(two120));
-    asm("mul.rn.bf16x2 %0, %1, %2;" : "=r"(hi) : "r"(b23), "r"(two120));
-}
-
-// One thread's share of widening a landed 8-bit tile [128 rows][64 bytes] into the bf16 tile of a compute stage: `items`
-// 16-byte groups starting at group `first + lane` and 32 apart.  Group g = 16 codes of row g / 4 (its quarter g % 4) -> the two
-// 16-byte chunks 2c, 2c + 1 of the bf16 row, each stored at chunk position (chunk ^ (row & 7)): the 128-byte swizzle the weight
-// tiles otherwise get from the copy engine.  Waits (bounded) for the tile and, when given, for the stage to be free.
-template <int ITEMS>
-__device__ __forceinline__ bool w8_convert_unit(const GemmParams &p, Barriers *bars, uint8_t *stage, const uint8_t *src, uint64_t *landed, uint32_t landed_parity,
-                                                uint64_t *stage_free, uint32_t free_parity, int first, int lane, int code) {
-    int good = 1;
-    if (lane == 0) {
-        good = ptx::mbar_wait_bounded(landed, landed_parity) ? 1 : 0;
-        if (good && stage_free) good = ptx::mbar_wait_bounded(stage_free, free_parity) ? 1 : 0;
-        if (!good) fail(p, bars, code);
-    }
-    good = __shfl_sync(0xffffffffu, good, 0);
-    if (!good) return false;
-    uint4 wv[ITEMS]; // (all reads first: the compiler cannot move them across the stores itself)
-#pragma unroll
-    for (int it = 0; it < ITEMS; ++it) wv[it] = *reinterpret_cast<const uint4 *>(src + (first + it * 32 + lane) * 16);
-#pragma unroll
-    for (int it = 0; it < ITEMS; ++it) {
-        const int idx = first + it * 32 + lane, r = idx >> 2, c = idx & 3;
-        const uint4 w = wv[it];
-        uint4 lo4, hi4;
-        e4m3x4_to_bf16x4(w.x, lo4.x, lo4.y); e4m3x4_to_bf16x4(w.y, lo4.z, lo4.w);
-        e4m3x4_to_bf16x4(w.z, hi4.x, hi4.y); e4m3x4_to_bf16x4(w.w, hi4.z, hi4.w);
-        uint8_t *row = stage + r * 128;
-        *reinterpret_cast<uint4 *>(row + (((2 * c) ^ (r & 7)) << 4)) = lo4;
-        *reinterpret_cast<uint4 *>(row + (((2 * c + 1) ^ (r & 7)) << 4)) = hi4;
-    }
-    ptx::fence_proxy_async_smem(); // the tensor cores read the tile through the asynchronous proxy
-    __syncwarp();
-    return true;
-}
-
-// The same for a tile that landed in the upper half of the stage's own bf16 buffer [128 rows][128 bytes]: the four epilogue warps
-// (`t` = 0..127) first read the whole 8-bit tile into registers, meet, and then write the bf16 tile over it.
-__device__ __forceinline__ bool w8_convert_in_place(const GemmParams &p, Barriers *bars, uint8_t *stage, uint64_t *landed, uint64_t *full, int t, int lane,
-                                                    int code) {
-    int good = 1;
-    if (lane == 0) {
-        good = ptx::mbar_wait_bounded(landed, 0) ? 1 : 0;
-        if (!good) fail(p, bars, code);
-    }
-    good = __shfl_sync(0xffffffffu, good, 0);
-    const uint8_t *src = stage + A8_BYTES;
-    uint4 w[4];
-#pragma unroll
-    for (int it = 0; it < 4; ++it)
-        if (good) w[it] = *reinterpret_cast<const uint4 *>(src + (t + it * 128) * 16);
-    asm volatile("bar.sync 3, 128;" ::: "memory"); // (a warp whose wait failed still meets the others here; they see the abort flag below)
-    if (!good || bars->abort) return false;
-#pragma unroll
-    for (int it = 0; it < 4; ++it) {
-        const int idx = t + it * 128, r = idx >> 2, c = idx & 3;
-        {
-            uint4 lo4, hi4;
-            e4m3x4_to_bf16x4(w[it].x, lo4.x, lo4.y); e4m3x4_to_bf16x4(w[it].y, lo4.z, lo4.w);
-            e4m3x4_to_bf16x4(w[it].z, hi4.x, hi4.y); e4m3x4_to_bf16x4(w[it].w, hi4.z, hi4.w);
-            uint8_t *row = stage + r * 128;
-            *reinterpret_cast<uint4 *>(row + (((2 * c) ^ (r & 7)) << 4)) = lo4;
-            *reinterpret_cast<uint4 *>(row + (((2 * c + 1) ^ (r & 7)) << 4)) = hi4;
-        }
-    }
-    ptx::fence_proxy_async_smem();
-    __syncwarp();
-    if (lane == 0) ptx::mbar_arrive(full);
-    return true;
-}
-
 // (Few enough registers for three CTAs of it, or two next to the element-wise kernels' CTAs, to be resident on an SM.)
 template <bool W8>
-__global__ void __launch_bounds__(W8 ? 640 : GEMM_THREADS, W8 ? 1 : 3) // (W8: bounds that cap it at 96 registers, like the bf16 instance)
-
+__global__ void __launch_bounds__(GEMM_THREADS, 3)
 gemm_ws_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant__ CUtensorMap map_hi,
                const __grid_constant__ CUtensorMap map_lo, const GemmParams p) {
     extern __shared__ uint8_t smem_raw[];
     // stage ring first (1024-byte aligned for the 128-byte swizzle), barriers after it
     uint8_t *smem = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
-    const int b_bytes = p.n_pad * TILE_K * 2;
-    const int stage_bytes = A_BYTES + b_bytes * (p.use_lo ? 2 : 1);
-    uint8_t *landing = smem + (size_t)p.stages * stage_bytes;     // W8: p.landing slots of A8_BYTES
-    Barriers *bars = reinterpret_cast<Barriers *>(landing + (W8 ? (size_t)p.landing * A8_BYTES : 0));
+    const int b_bytes = p.n_pad * TILE_K * 2;   // one activation plane of a stage: n_pad rows of 128 bytes (64 bf16 or 128 codes)
+    const int stage_bytes = A_BYTES + b_bytes * (W8 ? p.planes : p.use_lo ? 2 : 1);
+    constexpr int KT = W8 ? 2 * TILE_K : TILE_K; // elements of K per stage
+    Barriers *bars = reinterpret_cast<Barriers *>(smem + (size_t)p.stages * stage_bytes);
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     // this CTA's contiguous range of (tile, k tile) units
@@ -219,21 +126,19 @@ gemm_ws_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant_
     // The hi and lo planes of the activations are adjacent in a stage, so while 2 * n_pad <= 256 ONE MMA
     // covers both (N = 2 * n_pad, the lo part lands in its own accumulator columns and is added in the
     // epilogue): a tcgen05.mma costs about the same whatever N is, so this halves the tensor-pipe time.
-    const bool stacked = p.use_lo && 2 * p.n_pad <= 256;
-    const int acc_cols = stacked ? 2 * p.n_pad : p.n_pad;   // columns of one accumulator buffer
+    const bool stacked = !W8 && p.use_lo && 2 * p.n_pad <= 256;
+    const int acc_cols = W8 ? p.planes * p.n_pad : stacked ? 2 * p.n_pad : p.n_pad;   // columns of one accumulator buffer
     // two accumulator buffers, so that the epilogue of one output tile overlaps the MMAs of the next - unless the CTA
     // works on a single tile (tile-aligned split): then one buffer, and more CTAs' accumulators fit the SM's tensor memory
-    const uint32_t tmem_need = (p.split > 0 ? 1u : 2u) * acc_cols;
+    // (or two would not fit the 512 columns)
+    const int n_acc = (p.split > 0 || 2 * acc_cols > 512) ? 1 : 2;
+    const uint32_t tmem_need = (uint32_t)(n_acc * acc_cols);
     const uint32_t tmem_cols = tmem_need <= 32 ? 32u : tmem_need <= 64 ? 64u : tmem_need <= 128 ? 128u : tmem_need <= 256 ? 256u : 512u;
 
     ptx::pdl_launch_dependents(); // the next kernel may start: its CTAs begin their own weight prefetch as SMs have room
     if (threadIdx.x == 0) {
         ptx::trace_mark(p.trace, 0);
-        // (W8: a stage is full when its activations have landed and the converters have arrived: the four epilogue warps when
-        //  tiles land inside their stages; with the landing ring six warps' worth - six warps' one each, or the two dedicated
-        //  warps' three each)
-        for (int s = 0; s < p.stages; ++s) { ptx::mbar_init(&bars->full[s], W8 ? (p.landing ? 7 : 5) : 1); ptx::mbar_init(&bars->empty[s], 1); }
-        if (W8) for (int l = 0; l < max(p.landing, p.stages); ++l) { ptx::mbar_init(&bars->wfull[l], 1); ptx::mbar_init(&bars->wempty[l], 6); }
+        for (int s = 0; s < p.stages; ++s) { ptx::mbar_init(&bars->full[s], 1); ptx::mbar_init(&bars->empty[s], 1); }
         for (int a = 0; a < 2; ++a) { ptx::mbar_init(&bars->acc_full[a], 1); ptx::mbar_init(&bars->acc_empty[a], 4); }
         // a device error recorded by an earlier kernel makes every later one a no-op, so that a
         // failure costs one time-out, not one per launch
@@ -243,20 +148,14 @@ gemm_ws_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant_
         // They depend neither on the previous kernel nor on this CTA's tensor memory, whose allocation (below) waits
         // while the CTAs of the previous projection still hold theirs - with more than 32 nodes two CTAs fill it.
         if (!bars->abort && u1 > u0) {
-            if (!W8) ptx::prefetch_tensormap(&map_w);
+            ptx::prefetch_tensormap(&map_w);
             const uint64_t pol = ptx::policy_evict_first();
             const uint32_t tx = (uint32_t)stage_bytes;
             int tile = u0 / p.k_tiles, kt = u0 - tile * p.k_tiles;
-            const int pre = min(u1 - u0, (W8 && p.landing) ? p.landing : p.stages);
+            const int pre = min(u1 - u0, p.stages);
             for (int j = 0; j < pre; ++j) {
-                if (W8) {
-                    uint8_t *dst = p.landing ? landing + (size_t)j * A8_BYTES : smem + (size_t)j * stage_bytes + A8_BYTES;
-                    ptx::mbar_arrive_expect_tx(&bars->wfull[j], A8_BYTES);
-                    ptx::bulk_load_hint(dst, p.w_codes + (size_t)(u0 + j) * A8_BYTES, A8_BYTES, &bars->wfull[j], pol);
-                } else {
-                    ptx::mbar_arrive_expect_tx(&bars->full[j], tx);
-                    ptx::tma_load_2d_hint(smem + (size_t)j * stage_bytes, &map_w, kt * TILE_K, tile * TILE_M, &bars->full[j], pol);
-                }
+                ptx::mbar_arrive_expect_tx(&bars->full[j], tx);
+                ptx::tma_load_2d_hint(smem + (size_t)j * stage_bytes, &map_w, kt * KT, tile * TILE_M, &bars->full[j], pol);
                 if (++kt == p.k_tiles) { kt = 0; ++tile; }
             }
         }
@@ -277,11 +176,11 @@ gemm_ws_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant_
         // ===================== TMA producer =====================
         if (lane == 0 && u1 > u0) {
             ptx::prefetch_tensormap(&map_hi);
-            if (p.use_lo) ptx::prefetch_tensormap(&map_lo);
+            if (!W8 && p.use_lo) ptx::prefetch_tensormap(&map_lo);
             const uint64_t pol = ptx::policy_evict_first();
             const uint32_t tx = (uint32_t)stage_bytes;
             // (phase 1, the weight tiles of the first `pre` units, was issued before the CTA-wide set-up barrier)
-            const int pre = W8 ? 0 : min(u1 - u0, p.stages); // (W8: this thread loads activations only; the converters refill the landing slots)
+            const int pre = min(u1 - u0, p.stages);
             // (one integer division per role, none per unit: for one thread a division is ~150 cycles, and several per unit
             //  used to cost more than the unit's loads and tensor-core instructions)
             int tile = u0 / p.k_tiles, kt = u0 - tile * p.k_tiles, s = 0, round = 0;
@@ -291,31 +190,33 @@ gemm_ws_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant_
             for (int u = u0; u < u1 && ok; ++u) {
                 const int j = u - u0;
                 uint8_t *st = smem + (size_t)s * stage_bytes;
-                if (W8) {
-                    if (round > 0 && !ptx::mbar_wait_bounded(&bars->empty[s], (round - 1) & 1)) { fail(p, bars, 0x100 + s); ok = false; break; }
-                    ptx::mbar_arrive_expect_tx(&bars->full[s], (uint32_t)(stage_bytes - A_BYTES)); // the activation planes' bytes
-                } else if (j >= pre) {
+                if (j >= pre) {
                     if (!ptx::mbar_wait_bounded(&bars->empty[s], (round - 1) & 1)) { fail(p, bars, 0x100 + s); ok = false; break; }
                     ptx::mbar_arrive_expect_tx(&bars->full[s], tx);
-                    ptx::tma_load_2d_hint(st, &map_w, kt * TILE_K, tile * TILE_M, &bars->full[s], pol);
+                    ptx::tma_load_2d_hint(st, &map_w, kt * KT, tile * TILE_M, &bars->full[s], pol);
                 }
-                // (the activation maps' box is the whole padded batch: one operation per plane)
-                ptx::tma_load_2d(st + A_BYTES, &map_hi, kt * TILE_K, 0, &bars->full[s]);
-                if (p.use_lo) ptx::tma_load_2d(st + A_BYTES + b_bytes, &map_lo, kt * TILE_K, 0, &bars->full[s]);
+                // (the activation maps' box is the whole padded batch: one operation per plane; W8: one for the four planes)
+                if (W8) {
+                    ptx::tma_load_3d(st + A_BYTES, &map_hi, kt * KT, p.row0, 0, &bars->full[s]);
+                } else {
+                    ptx::tma_load_2d(st + A_BYTES, &map_hi, kt * TILE_K, 0, &bars->full[s]);
+                    if (p.use_lo) ptx::tma_load_2d(st + A_BYTES + b_bytes, &map_lo, kt * TILE_K, 0, &bars->full[s]);
+                }
                 if (bars->abort) ok = false;
                 if (++kt == p.k_tiles) { kt = 0; ++tile; }
                 if (++s == p.stages) { s = 0; ++round; }
             }
             if (!ok) {
                 // a failed wait: let the copies already in flight land before shared memory is released
-                if (W8) for (int l = 0; l < max(p.landing, p.stages); ++l) ptx::mbar_wait_bounded(&bars->wfull[l], 0, 20000000ll);
-                else for (int s = 0; s < p.stages; ++s) ptx::mbar_wait_bounded(&bars->full[s], 0, 20000000ll);
+                for (int s = 0; s < p.stages; ++s) ptx::mbar_wait_bounded(&bars->full[s], 0, 20000000ll);
             }
         }
     } else if (warp == 1) {
         // ===================== MMA issuer =====================
         if (lane == 0) {
-            const uint32_t idesc = ptx::umma_idesc_bf16(TILE_M, acc_cols);
+            // (W8: the stacked planes are 4 n_pad rows of B; an instruction takes at most 256 of them)
+            const int n_mma = (W8 && acc_cols > 256) ? 2 : 1, mma_n = acc_cols / n_mma;
+            const uint32_t idesc = W8 ? ptx::umma_idesc_e4m3(TILE_M, mma_n) : ptx::umma_idesc_bf16(TILE_M, mma_n);
             int seg = 0;
             bool ok = true;
             int kt = u0 % p.k_tiles, s = 0, round = 0; // (kept incrementally: no integer division inside the loop)
@@ -323,9 +224,9 @@ gemm_ws_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant_
                 const int j = u - u0;
                 const bool seg_first = (u == u0) || (kt == 0);
                 const bool seg_last = (u + 1 == u1) || (kt + 1 == p.k_tiles);
-                const int ab = seg & 1;
-                if (seg_first && seg >= 2) { // accumulator buffer reuse: wait until the epilogue drained it
-                    if (!ptx::mbar_wait_bounded(&bars->acc_empty[ab], ((seg >> 1) - 1) & 1)) { fail(p, bars, 0x200 + ab); ok = false; break; }
+                const int ab = n_acc == 2 ? seg & 1 : 0, use = n_acc == 2 ? seg >> 1 : seg; // buffer, and how often it was used before
+                if (seg_first && use >= 1) { // accumulator buffer reuse: wait until the epilogue drained it
+                    if (!ptx::mbar_wait_bounded(&bars->acc_empty[ab], (use - 1) & 1)) { fail(p, bars, 0x200 + ab); ok = false; break; }
                     ptx::tc_fence_after_sync();
                 }
                 if (!ptx::mbar_wait_bounded(&bars->full[s], round & 1)) { fail(p, bars, 0x300 + s); ok = false; break; }
@@ -335,10 +236,15 @@ gemm_ws_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant_
                 const uint32_t b_addr = a_addr + A_BYTES;
                 const uint32_t d_addr = tmem_base + (uint32_t)(ab * acc_cols);
 #pragma unroll
-                for (int k = 0; k < TILE_K / UMMA_K; ++k) {
+                for (int k = 0; k < TILE_K / UMMA_K; ++k) { // (four slices of 32 bytes of K, for either kind)
                     const uint64_t da = ptx::umma_desc_k_sw128(a_addr + k * UMMA_K * 2);
-                    ptx::umma_bf16(d_addr, da, ptx::umma_desc_k_sw128(b_addr + k * UMMA_K * 2), idesc, (seg_first && k == 0) ? 0u : 1u);
-                    if (p.use_lo && !stacked) ptx::umma_bf16(d_addr, da, ptx::umma_desc_k_sw128(b_addr + b_bytes + k * UMMA_K * 2), idesc, 1u);
+                    if (W8) {
+                        for (int g = 0; g < n_mma; ++g)
+                            ptx::umma_e4m3(d_addr + g * mma_n, da, ptx::umma_desc_k_sw128(b_addr + g * mma_n * 128 + k * 32), idesc, (seg_first && k == 0) ? 0u : 1u);
+                    } else {
+                        ptx::umma_bf16(d_addr, da, ptx::umma_desc_k_sw128(b_addr + k * UMMA_K * 2), idesc, (seg_first && k == 0) ? 0u : 1u);
+                        if (p.use_lo && !stacked) ptx::umma_bf16(d_addr, da, ptx::umma_desc_k_sw128(b_addr + b_bytes + k * UMMA_K * 2), idesc, 1u);
+                    }
                 }
                 if (j + p.stages < u1 - u0) ptx::umma_commit(&bars->empty[s]); // hand the stage back (only if a later unit of this CTA reuses it)
                 if (seg_last) { ptx::umma_commit(&bars->acc_full[ab]); ++seg; }
@@ -347,53 +253,9 @@ gemm_ws_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant_
                 if (++s == p.stages) { s = 0; ++round; }
             }
         }
-    } else if (W8 && warp >= 6) {
-        // ===================== dedicated converters (W8 with the landing ring: warps 6..13, four pairs) =====================
-        // A warp alone runs the dependent bit operations of a tile at a fraction of an instruction per cycle, so the pairs work
-        // on several units at once.  Pair q OWNS stage q: it widens units q, q + stages, ... one after the other, so that its
-        // parity waits on the stage's barriers always concern the phase next to the one it last saw (a pair that skipped ahead
-        // over a stage's phase would take an older phase of the same parity for the one it waits for).
-        const int pair = (warp - 6) >> 1, half = (warp - 6) & 1, n_units = u1 - u0;
-        const int helped = min(n_units, p.stages); // units the epilogue warps help with
-        const uint64_t pol = ptx::policy_evict_first();
-        for (int j = pair, round = 0; j < n_units && pair < p.stages; j += p.stages, ++round) {
-            const int s = pair, l = j % p.landing, lround = j / p.landing;
-            const bool with_help = j < helped;
-            uint8_t *st = smem + (size_t)s * stage_bytes;
-            const uint8_t *src = landing + (size_t)l * A8_BYTES;
-            const bool done = with_help ? w8_convert_unit<2>(p, bars, st, src, &bars->wfull[l], lround & 1, nullptr, 0, half * 64, lane, 0x500 + l)
-                                        : w8_convert_unit<8>(p, bars, st, src, &bars->wfull[l], lround & 1, round > 0 ? &bars->empty[s] : nullptr,
-                                                             (round - 1) & 1, half * 256, lane, 0x500 + l);
-            if (!done) break;
-            if (lane == 0) { // (unhelped units: the pair arrives for all six)
-                ptx::mbar_arrive_n(&bars->full[s], with_help ? 1u : 3u);
-                ptx::mbar_arrive_n(&bars->wempty[l], with_help ? 1u : 3u);
-                if (half == 0 && j + p.landing < n_units) { // the slot is read: request the unit that lands in it next
-                    if (!ptx::mbar_wait_bounded(&bars->wempty[l], lround & 1)) { fail(p, bars, 0x600 + l); }
-                    else {
-                        ptx::mbar_arrive_expect_tx(&bars->wfull[l], A8_BYTES);
-                        ptx::bulk_load_hint(landing + (size_t)l * A8_BYTES, p.w_codes + (size_t)(u0 + j + p.landing) * A8_BYTES, A8_BYTES, &bars->wfull[l], pol);
-                    }
-                }
-            }
-            __syncwarp();
-            if (bars->abort) break;
-        }
-        if (bars->abort && warp == 6 && lane == 0) // a failed wait somewhere: let the weight copies in flight land before shared memory is released
-            for (int q = 0; q < max(p.landing, p.stages); ++q) { ptx::mbar_wait_bounded(&bars->wfull[q], 0, 10000000ll); ptx::mbar_wait_bounded(&bars->wfull[q], 1, 10000000ll); }
     } else {
         // ===================== epilogue (warps 2..5) =====================
         const int quarter = warp & 3; // TMEM lanes a warp may touch: 32 * (warp id % 4) ...
-        if (W8) { // help to widen the CTA's first units (rows 32..127; the dedicated warps take rows 0..31): no epilogue is due before them
-            const int helped = min(u1 - u0, p.stages);
-            for (int j = 0; j < helped && p.landing == 0; ++j)
-                if (!w8_convert_in_place(p, bars, smem + (size_t)j * stage_bytes, &bars->wfull[j], &bars->full[j], threadIdx.x - 64, lane, 0x700 + j)) break;
-            for (int j = 0; j < helped && p.landing; ++j) // (there are at least as many landing slots as stages)
-                if (!w8_convert_unit<3>(p, bars, smem + (size_t)j * stage_bytes, landing + (size_t)j * A8_BYTES, &bars->wfull[j], 0, nullptr, 0,
-                                        128 + (warp - 2) * 96, lane, 0x700 + j))
-                    break;
-                else if (lane == 0) { ptx::mbar_arrive_n(&bars->full[j], 1u); ptx::mbar_arrive_n(&bars->wempty[j], 1u); }
-        }
         ptx::pdl_grid_wait();         // Y may still be read or written by the previous kernels
         float *const y = p.y ? p.y : p.info->logits;
         const int et = threadIdx.x - 64; // 0..127 among the epilogue threads
@@ -403,7 +265,7 @@ gemm_ws_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant_
             const int tile = u / p.k_tiles;
             const int seg_end = min(u1, (tile + 1) * p.k_tiles);
             const bool has_k0 = (u % p.k_tiles) == 0;
-            const int ab = seg & 1;
+            const int ab = n_acc == 2 ? seg & 1 : 0, use = n_acc == 2 ? seg >> 1 : seg;
             // (what does not depend on the accumulator is fetched before waiting for it)
             const int o = tile * TILE_M + quarter * 32 + lane;
             const float bias = (has_k0 && p.bias && o < p.out) ? p.bias[o] : 0.f;
@@ -411,13 +273,36 @@ gemm_ws_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant_
             const uint32_t taddr = tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(ab * acc_cols);
             // one lane per warp polls (spinning threads would compete with the tensor cores for shared memory)
             int good = ok ? 1 : 0;
-            if (lane == 0 && good) good = ptx::mbar_wait_bounded<EPI_POLL_NS>(&bars->acc_full[ab], (seg >> 1) & 1) ? 1 : 0;
+            if (lane == 0 && good) good = ptx::mbar_wait_bounded<EPI_POLL_NS>(&bars->acc_full[ab], use & 1) ? 1 : 0;
             good = __shfl_sync(0xffffffffu, good, 0);
             if (!good) { if (lane == 0) fail(p, bars, 0x400 + ab); ok = false; }
             if (seg == 0 && et == 0) ptx::trace_mark(p.trace, 3); // first accumulator complete
             ptx::tc_fence_after_sync();
             int warp_bad = 0;
-            for (int c0 = 0; c0 < p.n_pad && good; c0 += 16) {
+            if (W8) { // the planes' products of sixteen rows at a time: acc = 16 a0 + a1 + a2 / 16 + a3 / 256, times the row's scale
+                // (draining the accumulator is what this epilogue takes its time for - tensor memory reads at a fixed rate per SM - so
+                //  every plane left out shortens it)
+                for (int c0 = 0; c0 < p.n_pad && good; c0 += 16) { // (the loads are warp-wide: every lane runs the loop)
+                    uint32_t a0[16], a1[16], a2[16], a3[16];
+                    ptx::tmem_ld_32x16(taddr + c0, a0);
+                    ptx::tmem_ld_32x16(taddr + p.n_pad + c0, a1);
+                    if (p.planes > 2) ptx::tmem_ld_32x16(taddr + 2 * p.n_pad + c0, a2);
+                    if (p.planes > 3) ptx::tmem_ld_32x16(taddr + 3 * p.n_pad + c0, a3);
+                    ptx::tmem_ld_wait();
+                    if (o < p.out) {
+                        float *yo = y + (size_t)(p.row0 + c0) * p.ldy + o;
+                        const int rows = min(16, p.n - c0);
+#pragma unroll
+                        for (int t = 0; t < 16; ++t, yo += p.ldy) {
+                            const float hi = fmaf(16.f, __uint_as_float(a0[t]), __uint_as_float(a1[t]));
+                            float lo = p.planes > 2 ? __uint_as_float(a2[t]) : 0.f;
+                            if (p.planes > 3) lo = fmaf(0.0625f, __uint_as_float(a3[t]), lo);
+                            if (t < rows) ptx::red_add_f32(yo, fmaf(fmaf(0.0625f, lo, hi), scale, bias));
+                        }
+                    }
+                }
+            }
+            for (int c0 = 0; c0 < p.n_pad && good && !W8; c0 += 16) {
                 uint32_t r[16], q[16];
                 ptx::tmem_ld_32x16(taddr + c0, r);
                 if (stacked) ptx::tmem_ld_32x16(taddr + p.n_pad + c0, q); // the lo plane's part of the product
@@ -426,7 +311,7 @@ gemm_ws_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant_
                     float v[16];
 #pragma unroll
                     for (int t = 0; t < 16; ++t) {
-                        v[t] = (__uint_as_float(r[t]) + (stacked ? __uint_as_float(q[t]) : 0.f)) * scale + bias;
+                        v[t] = __uint_as_float(r[t]) + (stacked ? __uint_as_float(q[t]) : 0.f) + bias;
                         if (o < p.out && c0 + t < p.n) y[(size_t)(c0 + t) * p.ldy + o] = v[t];
                     }
                     if (p.stat_val) {
@@ -451,13 +336,13 @@ gemm_ws_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant_
                     float *yo = y + (size_t)c0 * p.ldy + o;
                     if (stacked && c0 + 16 <= p.n) { // the usual case, kept short: sixteen full rows, hi + lo columns
 #pragma unroll
-                        for (int t = 0; t < 16; ++t, yo += p.ldy) ptx::red_add_f32(yo, (__uint_as_float(r[t]) + __uint_as_float(q[t])) * scale + bias);
+                        for (int t = 0; t < 16; ++t, yo += p.ldy) ptx::red_add_f32(yo, __uint_as_float(r[t]) + __uint_as_float(q[t]) + bias);
                     } else {
 #pragma unroll
                         for (int t = 0; t < 16; ++t) {
                             const int i = c0 + t;
                             if (i < p.n) {
-                                float v = (__uint_as_float(r[t]) + (stacked ? __uint_as_float(q[t]) : 0.f)) * scale + bias;
+                                float v = __uint_as_float(r[t]) + (stacked ? __uint_as_float(q[t]) : 0.f) + bias;
                                 ptx::red_add_f32(yo + (size_t)t * p.ldy, v);
                             }
                         }
@@ -529,10 +414,38 @@ int make_tensor_map_bf16(void *map_out, const void *base, uint64_t rows, uint64_
     return r == CUDA_SUCCESS ? SSD_OK : SSD_ERR_CUDA;
 }
 
+// 8-bit operands.  Weights: codes [rows, cols] row-major (cols a multiple of 64), boxes of [box_rows, 128 codes], 128-byte
+// swizzle; a box that reaches past the matrix reads zeros (cols need not be a multiple of 128).
+int make_tensor_map_u8(void *map_out, const void *base, uint64_t rows, uint64_t cols, uint32_t box_rows) {
+    EncodeTiledFn fn = encode_fn();
+    if (!fn) return SSD_ERR_CUDA;
+    cuuint64_t dims[2] = {cols, rows};
+    cuuint64_t strides[1] = {cols};
+    cuuint32_t box[2] = {2 * TILE_K, box_rows};
+    cuuint32_t estr[2] = {1, 1};
+    CUresult r = fn((CUtensorMap *)map_out, CU_TENSOR_MAP_DATA_TYPE_UINT8, 2, const_cast<void *>(base), dims, strides, box, estr,
+                    CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                    CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    return r == CUDA_SUCCESS ? SSD_OK : SSD_ERR_CUDA;
+}
+// Activations: four planes [4][rows][cols] of codes; ONE box takes [the first box_planes planes][box_rows][128 codes].
+int make_tensor_map_u8_planes(void *map_out, const void *base, uint64_t rows, uint64_t cols, uint32_t box_rows, uint32_t box_planes) {
+    EncodeTiledFn fn = encode_fn();
+    if (!fn) return SSD_ERR_CUDA;
+    cuuint64_t dims[3] = {cols, rows, W8_PLANES};
+    cuuint64_t strides[2] = {cols, rows * cols};
+    cuuint32_t box[3] = {2 * TILE_K, box_rows, box_planes};
+    cuuint32_t estr[3] = {1, 1, 1};
+    CUresult r = fn((CUtensorMap *)map_out, CU_TENSOR_MAP_DATA_TYPE_UINT8, 3, const_cast<void *>(base), dims, strides, box, estr,
+                    CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                    CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    return r == CUDA_SUCCESS ? SSD_OK : SSD_ERR_CUDA;
+}
+
 // Pipeline depth.  With `shared_sm` (more CTAs than SMs) a CTA takes at most half an SM's shared memory, so that two
 // are resident and one's tensor-core and epilogue phases overlap the other's loads.
-int gemm_ws_stages(int n_pad, int use_lo, bool shared_sm) {
-    const int stage_bytes = A_BYTES + n_pad * TILE_K * 2 * (use_lo ? 2 : 1);
+int gemm_ws_stages(int n_pad, int planes, bool shared_sm) {
+    const int stage_bytes = A_BYTES + n_pad * TILE_K * 2 * planes;
     int s = (shared_sm ? SMEM_BUDGET_SHARED : SMEM_BUDGET) / stage_bytes;
     return s > MAX_STAGES ? MAX_STAGES : (s < 2 ? 2 : s);
 }
@@ -547,15 +460,17 @@ cudaError_t gemm_ws_prepare() {
 
 cudaError_t launch_gemm_ws(const void *map_w, const void *map_hi, const void *map_lo, float *y, const StepInfo *info, int ldy,
                            const float *bias, int n, int K, int out, int use_lo, int grid, int sm_count, int32_t *status, bool pdl,
-                           cudaStream_t s, unsigned long long *trace, const GemmHeadStats *head, const float *w_scale, const uint8_t *w_codes) {
+                           cudaStream_t s, unsigned long long *trace, const GemmHeadStats *head, const float *w_scale, int row0, int w8_planes) {
+    const bool w8 = w_scale != nullptr; // map_w: the codes; map_hi: the four activation planes
+    if (w8 && (n > 128 || head || w8_planes < 2 || w8_planes > W8_PLANES)) return cudaErrorInvalidValue;
     GemmParams p;
     p.trace = trace;
     p.y = y; p.info = info; p.bias = bias; p.n = n; p.n_pad = (n + 15) & ~15;
-    p.out = out; p.ldy = ldy; p.k_tiles = K / TILE_K; p.n_tiles = (out + TILE_M - 1) / TILE_M;
-    p.use_lo = use_lo; p.status = status; p.w_scale = w_scale; p.w_codes = w_codes;
-    const bool w8 = w_codes != nullptr; // the weights are 8-bit codes stored tile by tile; map_w is not used
+    p.out = out; p.ldy = ldy; p.k_tiles = w8 ? (K + 2 * TILE_K - 1) / (2 * TILE_K) : K / TILE_K; p.n_tiles = (out + TILE_M - 1) / TILE_M;
+    p.use_lo = use_lo; p.status = status; p.w_scale = w_scale; p.row0 = row0; p.planes = w8_planes;
     p.store = 0; p.stat_val = nullptr; p.stat_arg = nullptr; p.stat_bad = nullptr;
-    const int stage_bytes = A_BYTES + p.n_pad * TILE_K * 2 * (use_lo ? 2 : 1);
+    const int planes = w8 ? w8_planes : use_lo ? 2 : 1;
+    const int stage_bytes = A_BYTES + p.n_pad * TILE_K * 2 * planes;
     const long long units = (long long)p.n_tiles * p.k_tiles;
     if (grid > units) grid = (int)units;
     int per_cta = (int)((units + grid - 1) / grid);
@@ -576,31 +491,15 @@ cudaError_t launch_gemm_ws(const void *map_w, const void *map_hi, const void *ma
         p.split = 1; grid = p.n_tiles; per_cta = p.k_tiles;
         p.store = 1; p.stat_val = head->val; p.stat_arg = head->arg; p.stat_bad = head->bad;
     }
-    p.stages = gemm_ws_stages(p.n_pad, use_lo, grid > sm_count);
+    p.stages = gemm_ws_stages(p.n_pad, planes, grid > sm_count);
     if (p.stages > per_cta) p.stages = per_cta < 1 ? 1 : per_cta;
-    p.landing = 0;
-    if (w8) {
-        // a short ring of compute stages (three cover the activation copy and the conversion ahead of the tensor cores), the
-        // rest of the budget as landing slots: they are what covers the HBM latency
-        int budget = (grid > sm_count ? SMEM_BUDGET_SHARED : SMEM_BUDGET);
-        const int half_sm = 113 * 1024 - (int)sizeof(Barriers) - 1024; // what lets two CTAs share an SM
-        if (grid > sm_count && budget > half_sm) budget = half_sm;
-        if (per_cta > p.stages) { // more units than stages: the landing ring (otherwise tiles land inside their stages)
-            if (p.stages > W8_PAIRS) p.stages = W8_PAIRS; // (one pair of converter warps per stage)
-            while (p.stages > 1 && p.stages * stage_bytes + p.stages * A8_BYTES > budget) --p.stages;
-            p.landing = (budget - p.stages * stage_bytes) / A8_BYTES;
-            if (p.landing > MAX_LANDING) p.landing = MAX_LANDING;
-            if (p.landing > per_cta) p.landing = per_cta;
-            if (p.landing < p.stages) p.landing = p.stages;
-        }
-    }
-    size_t smem = (size_t)p.stages * stage_bytes + (size_t)p.landing * A8_BYTES + sizeof(Barriers) + 1024;
+    size_t smem = (size_t)p.stages * stage_bytes + sizeof(Barriers) + 1024;
     // Two CTAs per SM, not three: with a third one resident the slowest CTA of a projection ends later (measured: 1.19 ms per
     // GPT-2-large verification of 32 nodes against 1.09 ms), so a CTA asks for more than a third of an SM's shared memory.
     if (grid > sm_count && smem < 78 * 1024) smem = 78 * 1024;
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3(grid);
-    cfg.blockDim = dim3(w8 && p.landing ? GEMM_THREADS_W8 : GEMM_THREADS);
+    cfg.blockDim = dim3(GEMM_THREADS);
     cfg.dynamicSmemBytes = smem;
     cfg.stream = s;
     cudaLaunchAttribute attr[1];
@@ -608,7 +507,6 @@ cudaError_t launch_gemm_ws(const void *map_w, const void *map_hi, const void *ma
     attr[0].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attr;
     cfg.numAttrs = pdl ? 1 : 0;
-    if (w8) map_w = map_hi;
     return cudaLaunchKernelEx(&cfg, w8 ? gemm_ws_kernel<true> : gemm_ws_kernel<false>, *(const CUtensorMap *)map_w,
                               *(const CUtensorMap *)map_hi, *(const CUtensorMap *)(map_lo ? map_lo : map_hi), p);
 }

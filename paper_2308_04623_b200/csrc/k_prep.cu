@@ -5,8 +5,12 @@
 // A value v is handed to the tensor cores as two bf16 planes, hi = bf16(v) and
 // lo = bf16(v - hi); the projection multiplies both by the same weight tile, which keeps the
 // activations to ~16 mantissa bits at no cost in HBM traffic.
+//
+// With 8-bit weights the projections run on the 8-bit tensor-core kind and read their activations as four e4m3 planes
+// instead (the P8 instantiations; see w8_planes.cuh).
 #include "sm100_ptx.cuh"
 #include "ssd_internal.h"
+#include "w8_planes.cuh"
 
 namespace {
 __device__ __forceinline__ float block_sum_256(float v, float *red) {
@@ -29,11 +33,12 @@ __device__ __forceinline__ uint2 pack4_bf16(float a, float b, float c, float d) 
     const __nv_bfloat162 lo = __floats2bfloat162_rn(a, b), hi = __floats2bfloat162_rn(c, d);
     return make_uint2(*reinterpret_cast<const uint32_t *>(&lo), *reinterpret_cast<const uint32_t *>(&hi));
 }
-template <int PER4>
+template <int PER4, bool P8>
 __global__ void __launch_bounds__(256) ln_prep_kernel(const float *__restrict__ x, const float *__restrict__ g, const float *__restrict__ b,
                                                       int d, float eps, __nv_bfloat16 *__restrict__ a_hi, __nv_bfloat16 *__restrict__ a_lo,
                                                       float *__restrict__ zero, int zero_cols, const StepInfo *__restrict__ info,
-                                                      int zero_from_info, unsigned long long *trace) {
+                                                      int zero_from_info, unsigned long long *trace, uint8_t *__restrict__ planes8,
+                                                      size_t plane_stride) {
     __shared__ float red[8];
     if (threadIdx.x == 0) ptx::trace_mark(trace, 0);
     ptx::pdl_launch_dependents();
@@ -74,8 +79,9 @@ __global__ void __launch_bounds__(256) ln_prep_kernel(const float *__restrict__ 
         if (k4 < d4) {
             const float o0 = v[q].x * rstd * gv[q].x + bv[q].x, o1 = v[q].y * rstd * gv[q].y + bv[q].y;
             const float o2 = v[q].z * rstd * gv[q].z + bv[q].z, o3 = v[q].w * rstd * gv[q].w + bv[q].w;
-            const uint2 hi = pack4_bf16(o0, o1, o2, o3);
             const size_t at = (size_t)i * d + 4 * (size_t)k4;
+            if (P8) { w8::store4(planes8, plane_stride, at, o0, o1, o2, o3); continue; }
+            const uint2 hi = pack4_bf16(o0, o1, o2, o3);
             *reinterpret_cast<uint2 *>(a_hi + at) = hi;
             if (a_lo) {
                 const float h0 = __uint_as_float(hi.x << 16), h1 = __uint_as_float(hi.x & 0xffff0000u);
@@ -102,8 +108,10 @@ __device__ __forceinline__ float gelu_tanh_fast(float z) { // 0.5 z (1 + tanh u)
     const float u2 = 1.5957691216057308f * (z + 0.044715f * z * z * z);
     return __fdividef(z, 1.0f + __expf(-u2));
 }
+template <bool P8>
 __global__ void __launch_bounds__(256) gelu_prep_kernel(const float *__restrict__ acc, size_t count, __nv_bfloat16 *__restrict__ h_hi,
-                                                        __nv_bfloat16 *__restrict__ h_lo, unsigned long long *trace) {
+                                                        __nv_bfloat16 *__restrict__ h_lo, unsigned long long *trace, uint8_t *__restrict__ planes8,
+                                                        size_t plane_stride) {
     if (threadIdx.x == 0) ptx::trace_mark(trace, 0);
     ptx::pdl_launch_dependents();
     ptx::pdl_grid_wait();
@@ -113,6 +121,11 @@ __global__ void __launch_bounds__(256) gelu_prep_kernel(const float *__restrict_
         float v[8] = {a.x, a.y, a.z, a.w, b.x, b.y, b.z, b.w};
 #pragma unroll
         for (int q = 0; q < 8; ++q) v[q] = gelu_tanh_fast(v[q]);
+        if (P8) { // (the flat index is row * F + k: the planes have the same shape)
+            w8::store4(planes8, plane_stride, e, v[0], v[1], v[2], v[3]);
+            w8::store4(planes8, plane_stride, e + 4, v[4], v[5], v[6], v[7]);
+            continue;
+        }
         const uint2 h0 = pack4_bf16(v[0], v[1], v[2], v[3]), h1 = pack4_bf16(v[4], v[5], v[6], v[7]);
         *reinterpret_cast<uint4 *>(h_hi + e) = make_uint4(h0.x, h0.y, h1.x, h1.y);
         if (h_lo) {
@@ -165,9 +178,11 @@ cudaError_t launch_pdl(void (*kernel)(Args...), dim3 grid, dim3 block, cudaStrea
 // All kernels of the forward ask for the same (maximum) shared-memory carve-out: an SM that has
 // to switch its L1/shared split between two kernels cannot overlap them.
 cudaError_t prep_kernels_prepare() {
-    cudaError_t e = cudaFuncSetAttribute(ln_prep_kernel<2>, cudaFuncAttributePreferredSharedMemoryCarveout, cudaSharedmemCarveoutMaxShared);
-    if (e == cudaSuccess) e = cudaFuncSetAttribute(ln_prep_kernel<8>, cudaFuncAttributePreferredSharedMemoryCarveout, cudaSharedmemCarveoutMaxShared);
-    if (e == cudaSuccess) e = cudaFuncSetAttribute(gelu_prep_kernel, cudaFuncAttributePreferredSharedMemoryCarveout, cudaSharedmemCarveoutMaxShared);
+    cudaError_t e = cudaSuccess;
+    const void *kernels[] = {(const void *)ln_prep_kernel<2, false>, (const void *)ln_prep_kernel<8, false>, (const void *)ln_prep_kernel<2, true>,
+                             (const void *)ln_prep_kernel<8, true>, (const void *)gelu_prep_kernel<false>, (const void *)gelu_prep_kernel<true>};
+    for (const void *k : kernels)
+        if (e == cudaSuccess) e = cudaFuncSetAttribute(k, cudaFuncAttributePreferredSharedMemoryCarveout, cudaSharedmemCarveoutMaxShared);
     return e;
 }
 
@@ -179,22 +194,22 @@ cudaError_t launch_ln_fold(const void *W, const float *g, const float *beta, con
 
 cudaError_t launch_ln_prep(const float *x, const float *g, const float *b, int n, int d, float eps, __nv_bfloat16 *a_hi, __nv_bfloat16 *a_lo,
                            float *zero, int zero_cols, const StepInfo *info, int zero_from_info, bool pdl, cudaStream_t s,
-                           unsigned long long *trace) {
+                           unsigned long long *trace, uint8_t *planes8, size_t plane_stride) {
     if ((d & 3) || d > 8192) return cudaErrorInvalidValue;
-    return launch_pdl(d <= 2048 ? ln_prep_kernel<2> : ln_prep_kernel<8>, dim3(n), dim3(256), s, pdl, x, g, b, d, eps, a_hi, a_lo, zero, zero_cols, info,
-                      zero_from_info, trace);
+    auto kernel = planes8 ? (d <= 2048 ? ln_prep_kernel<2, true> : ln_prep_kernel<8, true>) : (d <= 2048 ? ln_prep_kernel<2, false> : ln_prep_kernel<8, false>);
+    return launch_pdl(kernel, dim3(n), dim3(256), s, pdl, x, g, b, d, eps, a_hi, a_lo, zero, zero_cols, info, zero_from_info, trace, planes8, plane_stride);
 }
 
 cudaError_t launch_gelu_prep(const float *acc, int n, int F, __nv_bfloat16 *h_hi, __nv_bfloat16 *h_lo, bool pdl, cudaStream_t s,
-                             unsigned long long *trace) {
+                             unsigned long long *trace, uint8_t *planes8, size_t plane_stride) {
     const size_t count = (size_t)n * F;
     int grid = (int)((count + 256 * 8 - 1) / (256 * 8));
     if (grid > 148 * 4) grid = 148 * 4;
-    return launch_pdl(gelu_prep_kernel, dim3(grid), dim3(256), s, pdl, acc, count, h_hi, h_lo, trace);
+    return launch_pdl(planes8 ? gelu_prep_kernel<true> : gelu_prep_kernel<false>, dim3(grid), dim3(256), s, pdl, acc, count, h_hi, h_lo, trace, planes8,
+                      plane_stride);
 }
 
 // ---- 8-bit weights: per-row power-of-two scale and e4m3 codes (run once, when the model is loaded) ----
-#include <cuda_fp8.h>
 namespace {
 __global__ void __launch_bounds__(256) quantise_rows_e4m3_kernel(const __nv_bfloat16 *__restrict__ w, size_t cols, uint8_t *__restrict__ codes,
                                                                  float *__restrict__ scales) {
@@ -224,12 +239,9 @@ __global__ void __launch_bounds__(256) quantise_rows_e4m3_kernel(const __nv_bflo
     __syncthreads();
     const float inv = 1.f / scale_sh; // (a power of two: exact)
     for (size_t k = threadIdx.x; k < cols; k += blockDim.x)
-        codes[((row >> 7) * (cols >> 6) + (k >> 6)) * 8192 + (row & 127) * 64 + (k & 63)] =
-            (uint8_t)__nv_cvt_float_to_fp8(__bfloat162float(src[k]) * inv, __NV_SATFINITE, __NV_E4M3);
+        codes[row * cols + k] = (uint8_t)__nv_cvt_float_to_fp8(__bfloat162float(src[k]) * inv, __NV_SATFINITE, __NV_E4M3);
 }
 } // namespace
-
-size_t w8_tiled_bytes(size_t rows, size_t cols) { return ((rows + 127) / 128) * (cols / 64) * 8192; }
 
 cudaError_t launch_quantise_rows_e4m3(const void *w_bf16, size_t rows, size_t cols, uint8_t *codes, float *scales, cudaStream_t s) {
     quantise_rows_e4m3_kernel<<<(unsigned)rows, 256, 0, s>>>((const __nv_bfloat16 *)w_bf16, cols, codes, scales);

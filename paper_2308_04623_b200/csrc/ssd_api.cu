@@ -45,6 +45,9 @@ struct ssd_ctx {
     bool w8;                           // bf16 model whose five matrix families are held as e4m3 codes + per-row scales
     uint8_t *wte8;                     // w8: the output head's codes [vocab, d_model] (the embedding look-up keeps the bf16 table)
     float *wte_scale;
+    int w8_planes;                     // w8: how many of the four planes the projections use (the rest of a value is dropped)
+    uint8_t *a8, *o8, *h8;             // w8: activation operands as four e4m3 planes [4][plane_rows][d_model or d_ff] (ActMaps then holds their
+                                       // maps in a_hi / o_hi / h_hi)
     int use_lo, pdl, gemm_grid, head_grid, trace_kernels, trace_count, use_graph, use_cluster, cl_max, cl_size[4], attn_lo;
     // cluster-reduced path: per-layer vectors that fold a LayerNorm into the projection behind it (c1 = W gain,
     // c2 = W beta + bias), and the two row-statistics buffers [tile][SSD_MAX_NODES][2] (in front of QKV / of FC)
@@ -167,6 +170,14 @@ static const ssd_ctx::ActMaps *act_maps_pad(ssd_ctx *ctx, int n_pad) {
     ssd_ctx::ActMaps &am = ctx->act_maps[n_pad / 16 - 1];
     if (!am.built) {
         const size_t d = ctx->cfg.d_model, F = ctx->cfg.d_ff, rows = ctx->plane_rows;
+        if (ctx->w8) {
+            int m8 = make_tensor_map_u8_planes(&am.a_hi, ctx->a8, rows, d, n_pad, ctx->w8_planes);
+            if (m8 == SSD_OK) m8 = make_tensor_map_u8_planes(&am.o_hi, ctx->o8, rows, d, n_pad, ctx->w8_planes);
+            if (m8 == SSD_OK) m8 = make_tensor_map_u8_planes(&am.h_hi, ctx->h8, rows, F, n_pad, ctx->w8_planes);
+            if (m8 != SSD_OK) return nullptr;
+            am.built = true;
+            return &am;
+        }
         int m = make_tensor_map_bf16(&am.a_hi, ctx->a_hi, rows, d, n_pad);
         if (m == SSD_OK) m = make_tensor_map_bf16(&am.a_lo, ctx->a_lo, rows, d, n_pad);
         if (m == SSD_OK) m = make_tensor_map_bf16(&am.o_hi, ctx->o_hi, rows, d, n_pad);
@@ -187,8 +198,10 @@ static int gemm_grid_for(const ssd_ctx *ctx, int n) {
     if (ctx->gemm_grid > 0) return ctx->gemm_grid;
     return ((n + 15) & ~15) <= 64 ? 2 * ctx->sm_count : ctx->sm_count;
 }
-// (8-bit weights: one CTA per SM, whose landing ring is then deep enough to keep the HBM stream of the head busy)
-static int head_grid_for(const ssd_ctx *ctx, int n) { return ctx->head_grid > 0 ? ctx->head_grid : ctx->w8 ? ctx->sm_count : gemm_grid_for(ctx, n); }
+// (8-bit weights: four accumulator column groups per node; two CTAs' double-buffered accumulators fit an SM up to 32 nodes)
+static int head_grid_for(const ssd_ctx *ctx, int n) {
+    return ctx->head_grid > 0 ? ctx->head_grid : (ctx->w8 && n > 32) ? ctx->sm_count : gemm_grid_for(ctx, n);
+}
 
 // Timeline slots of the next launch (profiling aid, off by default).
 static unsigned long long *trace_slot(ssd_ctx *ctx, int kernels) {
@@ -210,7 +223,7 @@ cudaError_t enqueue_forward(ssd_ctx *ctx, int n, int cap, const NodeList &tk, co
     // The LM head either holds complete sums per CTA (plain stores, row statistics per tile) or adds stream-K partial sums
     // into logits cleared here, at the start of the forward.
     const GemmHeadStats head_stats = {ctx->head_val, ctx->head_arg, ctx->head_bad};
-    const GemmHeadStats *head = (ctx->tensor_path && ctx->use_head_stats) ? &head_stats : nullptr;
+    const GemmHeadStats *head = (ctx->tensor_path && ctx->use_head_stats && !ctx->w8) ? &head_stats : nullptr;
     if (ctx->tensor_path && !head) Q(launch_zero_logits(info, n, c.vocab, s));
     if (ctx->tensor_path && ctx->use_cluster && !ctx->w8 && gemm_cl_supports(n, c.d_model)) {
         // bf16 model, trees of up to 64 nodes: five launches per layer.  Every projection reduces its split-K partial sums
@@ -267,22 +280,55 @@ cudaError_t enqueue_forward(ssd_ctx *ctx, int n, int cap, const NodeList &tk, co
         // accumulate their stream-K partial sums into fp32 buffers; every kernel is a programmatic dependent launch.
         const bool pdl = ctx->pdl != 0;
         const int lo = ctx->use_lo, grid = gemm_grid_for(ctx, n), hgrid = head_grid_for(ctx, n), sms = ctx->sm_count;
-        const bool w8 = ctx->w8;
         __nv_bfloat16 *a_lo = lo ? ctx->a_lo : nullptr, *o_lo = lo ? ctx->o_lo : nullptr, *h_lo = lo ? ctx->h_lo : nullptr;
+        if (ctx->w8) {
+            // 8-bit weights: the same eight launches per layer; the element-wise kernels and the attention write four e4m3 planes,
+            // the projections run on the 8-bit tensor-core kind.  A projection takes at most 128 nodes (512 accumulator columns):
+            // a larger tree runs each projection as two launches over the two halves of the nodes.
+            const size_t rows = ctx->plane_rows, sa = rows * (size_t)d, sh = rows * (size_t)F;
+            const int n1 = n > 128 ? 128 : n, n2 = n - n1;
+            const ssd_ctx::ActMaps *m1 = act_maps_for(ctx, n1), *m2 = n2 ? act_maps_for(ctx, n2) : nullptr;
+            if (!m1 || (n2 && !m2)) return cudaErrorUnknown;
+            auto gemm8 = [&](const TensorMap *w, const TensorMap ssd_ctx::ActMaps::*act, float *y, int ldy, const float *bias, int K, int out, int g,
+                             const float *scale) -> cudaError_t {
+                cudaError_t e8 = launch_gemm_ws(w, &(m1->*act), nullptr, y, info, ldy, bias, n1, K, out, 0, g, sms, ctx->d_status, pdl, s, trace_slot(ctx, *kernels), nullptr, scale, 0, ctx->w8_planes);
+                if (e8 == cudaSuccess && n2) {
+                    ++*kernels;
+                    e8 = launch_gemm_ws(w, &(m2->*act), nullptr, y, info, ldy, bias, n2, K, out, 0, g, sms, ctx->d_status, pdl, s, trace_slot(ctx, *kernels), nullptr, scale, n1, ctx->w8_planes);
+                }
+                return e8;
+            };
+            for (int l = 0; l < c.n_layer; ++l) {
+                const LayerWeights &L = ctx->layers[l];
+                const TensorMap *t = &ctx->map_layers[(size_t)4 * l];
+                Q(launch_ln_prep(ctx->x, L.ln1_g, L.ln1_b, n, d, c.ln_eps, nullptr, nullptr, ctx->qkv, 3 * d, info, 0, pdl, s, trace_slot(ctx, *kernels), ctx->a8, sa));
+                Q(gemm8(&t[0], &ssd_ctx::ActMaps::a_hi, ctx->qkv, 3 * d, L.b_qkv, d, 3 * d, grid, L.s_qkv));
+                Q(launch_tree_attention_mma(ctx->qkv, info, l * layer_elems, ctx->meta, n, c.n_head, cap, nullptr, nullptr, pdl, s, trace_slot(ctx, *kernels), ctx->attn_lo != 0, ctx->o8, sa));
+                Q(gemm8(&t[1], &ssd_ctx::ActMaps::o_hi, ctx->x, d, L.b_o, d, d, grid, L.s_o));
+                Q(launch_ln_prep(ctx->x, L.ln2_g, L.ln2_b, n, d, c.ln_eps, nullptr, nullptr, ctx->h, F, info, 0, pdl, s, trace_slot(ctx, *kernels), ctx->a8, sa));
+                Q(gemm8(&t[2], &ssd_ctx::ActMaps::a_hi, ctx->h, F, L.b_fc, d, F, grid, L.s_fc));
+                Q(launch_gelu_prep(ctx->h, n, F, nullptr, nullptr, pdl, s, trace_slot(ctx, *kernels), ctx->h8, sh));
+                Q(gemm8(&t[3], &ssd_ctx::ActMaps::h_hi, ctx->x, d, L.b_proj, F, d, grid, L.s_proj));
+            }
+            Q(launch_ln_prep(ctx->x, ctx->lnf_g, ctx->lnf_b, n, d, c.ln_eps, nullptr, nullptr, nullptr, 0, info, 0, pdl, s, trace_slot(ctx, *kernels), ctx->a8, sa));
+            Q(gemm8(&ctx->map_wte, &ssd_ctx::ActMaps::a_hi, nullptr, c.vocab, nullptr, d, c.vocab, hgrid, ctx->wte_scale));
+            ctx->trace_count = ctx->trace_kernels ? 8 * *kernels : 0;
+            return cudaSuccess;
+        }
         for (int l = 0; l < c.n_layer; ++l) {
             const LayerWeights &L = ctx->layers[l];
             const TensorMap *t = &ctx->map_layers[(size_t)4 * l];
             Q(launch_ln_prep(ctx->x, L.ln1_g, L.ln1_b, n, d, c.ln_eps, ctx->a_hi, a_lo, ctx->qkv, 3 * d, info, 0, pdl, s, trace_slot(ctx, *kernels)));
-            Q(launch_gemm_ws(&t[0], &am->a_hi, &am->a_lo, ctx->qkv, info, 3 * d, L.b_qkv, n, d, 3 * d, lo, grid, sms, ctx->d_status, pdl, s, trace_slot(ctx, *kernels), nullptr, L.s_qkv, w8 ? (const uint8_t *)L.w_qkv : nullptr));
+            Q(launch_gemm_ws(&t[0], &am->a_hi, &am->a_lo, ctx->qkv, info, 3 * d, L.b_qkv, n, d, 3 * d, lo, grid, sms, ctx->d_status, pdl, s, trace_slot(ctx, *kernels)));
             Q(launch_tree_attention_mma(ctx->qkv, info, l * layer_elems, ctx->meta, n, c.n_head, cap, ctx->o_hi, o_lo, pdl, s, trace_slot(ctx, *kernels), ctx->attn_lo != 0));
-            Q(launch_gemm_ws(&t[1], &am->o_hi, &am->o_lo, ctx->x, info, d, L.b_o, n, d, d, lo, grid, sms, ctx->d_status, pdl, s, trace_slot(ctx, *kernels), nullptr, L.s_o, w8 ? (const uint8_t *)L.w_o : nullptr));
+            Q(launch_gemm_ws(&t[1], &am->o_hi, &am->o_lo, ctx->x, info, d, L.b_o, n, d, d, lo, grid, sms, ctx->d_status, pdl, s, trace_slot(ctx, *kernels)));
             Q(launch_ln_prep(ctx->x, L.ln2_g, L.ln2_b, n, d, c.ln_eps, ctx->a_hi, a_lo, ctx->h, F, info, 0, pdl, s, trace_slot(ctx, *kernels)));
-            Q(launch_gemm_ws(&t[2], &am->a_hi, &am->a_lo, ctx->h, info, F, L.b_fc, n, d, F, lo, grid, sms, ctx->d_status, pdl, s, trace_slot(ctx, *kernels), nullptr, L.s_fc, w8 ? (const uint8_t *)L.w_fc : nullptr));
+            Q(launch_gemm_ws(&t[2], &am->a_hi, &am->a_lo, ctx->h, info, F, L.b_fc, n, d, F, lo, grid, sms, ctx->d_status, pdl, s, trace_slot(ctx, *kernels)));
             Q(launch_gelu_prep(ctx->h, n, F, ctx->h_hi, h_lo, pdl, s, trace_slot(ctx, *kernels)));
-            Q(launch_gemm_ws(&t[3], &am->h_hi, &am->h_lo, ctx->x, info, d, L.b_proj, n, F, d, lo, grid, sms, ctx->d_status, pdl, s, trace_slot(ctx, *kernels), nullptr, L.s_proj, w8 ? (const uint8_t *)L.w_proj : nullptr));
+            Q(launch_gemm_ws(&t[3], &am->h_hi, &am->h_lo, ctx->x, info, d, L.b_proj, n, F, d, lo, grid, sms, ctx->d_status, pdl, s, trace_slot(ctx, *kernels)));
         }
         Q(launch_ln_prep(ctx->x, ctx->lnf_g, ctx->lnf_b, n, d, c.ln_eps, ctx->a_hi, a_lo, nullptr, 0, info, 0, pdl, s, trace_slot(ctx, *kernels)));
-        Q(launch_gemm_ws(&ctx->map_wte, &am->a_hi, &am->a_lo, nullptr, info, c.vocab, nullptr, n, d, c.vocab, lo, hgrid, sms, ctx->d_status, pdl, s, trace_slot(ctx, *kernels), head, ctx->wte_scale, ctx->wte8));
+        Q(launch_gemm_ws(&ctx->map_wte, &am->a_hi, &am->a_lo, nullptr, info, c.vocab, nullptr, n, d, c.vocab, lo, hgrid, sms, ctx->d_status, pdl, s, trace_slot(ctx, *kernels), head));
         ctx->trace_count = ctx->trace_kernels ? 8 * *kernels : 0;
     } else {
         for (int l = 0; l < c.n_layer; ++l) {
@@ -393,6 +439,7 @@ int ssd_create(const ssd_config *cfg, int device, void *cuda_stream, ssd_ctx **o
     ctx->w8 = cfg->dtype == SSD_DTYPE_BF16_W8;
     if (ctx->w8) ctx->cfg.dtype = SSD_DTYPE_BF16;
     ctx->wte8 = nullptr; ctx->wte_scale = nullptr;
+    ctx->w8_planes = 4;
     ctx->device = device;
     ctx->stream = (cudaStream_t)cuda_stream;
     ctx->loaded = false;
@@ -442,6 +489,8 @@ int ssd_create(const ssd_config *cfg, int device, void *cuda_stream, ssd_ctx **o
         const size_t rows = n <= 32 ? 32 : ((n + 15) & ~size_t(15)); // operand planes hold whole 16-row boxes, at least two
         A(&ctx->a_hi, rows * d); A(&ctx->a_lo, rows * d); A(&ctx->o_hi, rows * d); A(&ctx->o_lo, rows * d);
         A(&ctx->h_hi, rows * (size_t)cfg->d_ff); A(&ctx->h_lo, rows * (size_t)cfg->d_ff);
+        ctx->a8 = ctx->o8 = ctx->h8 = nullptr;
+        if (ctx->w8) { A(&ctx->a8, 4 * rows * d); A(&ctx->o8, 4 * rows * d); A(&ctx->h8, 4 * rows * (size_t)cfg->d_ff); }
         ctx->head_tiles = (cfg->vocab + 127) / 128;
         A(&ctx->head_val, n * (size_t)ctx->head_tiles); A(&ctx->head_arg, n * (size_t)ctx->head_tiles); A(&ctx->head_bad, n * (size_t)ctx->head_tiles);
         if (rc == SSD_OK) {
@@ -449,6 +498,9 @@ int ssd_create(const ssd_config *cfg, int device, void *cuda_stream, ssd_ctx **o
             __nv_bfloat16 *planes[6] = {ctx->a_hi, ctx->a_lo, ctx->o_hi, ctx->o_lo, ctx->h_hi, ctx->h_lo};
             for (int q = 0; q < 6 && e == cudaSuccess; ++q)
                 e = cudaMemsetAsync(planes[q], 0, rows * (q < 4 ? d : (size_t)cfg->d_ff) * sizeof(__nv_bfloat16), ctx->stream);
+            uint8_t *planes8[3] = {ctx->a8, ctx->o8, ctx->h8}; // (rows past the tree are read by the projections' boxes: zero codes)
+            for (int q = 0; q < 3 && e == cudaSuccess && ctx->w8; ++q)
+                e = cudaMemsetAsync(planes8[q], 0, 4 * rows * (q < 2 ? d : (size_t)cfg->d_ff), ctx->stream);
             int dev_sms = 0;
             if (e == cudaSuccess) e = cudaDeviceGetAttribute(&dev_sms, cudaDevAttrMultiProcessorCount, device);
             if (e == cudaSuccess) e = gemm_ws_prepare();
@@ -534,10 +586,9 @@ int ssd_load_weights(ssd_ctx *ctx, const ssd_weights *w) {
         auto quantise = [&](const void *src, size_t rows, size_t cols, const void **codes_out, const float **scales_out) -> int {
             uint8_t *q = nullptr;
             float *sc = nullptr;
-            int r = dev_alloc(ctx, &q, w8_tiled_bytes(rows, cols));
+            int r = dev_alloc(ctx, &q, rows * cols);
             if (r == SSD_OK) r = dev_alloc(ctx, &sc, rows);
             if (r != SSD_OK) return r;
-            CU(cudaMemsetAsync(q, 0, w8_tiled_bytes(rows, cols), ctx->stream));
             CU(launch_quantise_rows_e4m3(src, rows, cols, q, sc, ctx->stream));
             *codes_out = q; *scales_out = sc;
             return SSD_OK;
@@ -563,14 +614,15 @@ int ssd_load_weights(ssd_ctx *ctx, const ssd_weights *w) {
     }
     if (ctx->tensor_path) {
         ctx->map_layers.assign((size_t)4 * c.n_layer, TensorMap());
-        int m = ctx->w8 ? SSD_OK : make_tensor_map_bf16(&ctx->map_wte, ctx->wte, c.vocab, d, 128);
-        for (int l = 0; l < c.n_layer && m == SSD_OK && !ctx->w8; ++l) { // (8-bit codes are fetched as contiguous tiles: no maps)
+        auto make_map = ctx->w8 ? make_tensor_map_u8 : make_tensor_map_bf16;
+        int m = make_map(&ctx->map_wte, ctx->w8 ? (const void *)ctx->wte8 : ctx->wte, c.vocab, d, 128);
+        for (int l = 0; l < c.n_layer && m == SSD_OK; ++l) {
             const LayerWeights &L = ctx->layers[l];
             TensorMap *t = &ctx->map_layers[(size_t)4 * l];
-            m = make_tensor_map_bf16(&t[0], L.w_qkv, 3 * d, d, 128);
-            if (m == SSD_OK) m = make_tensor_map_bf16(&t[1], L.w_o, d, d, 128);
-            if (m == SSD_OK) m = make_tensor_map_bf16(&t[2], L.w_fc, F, d, 128);
-            if (m == SSD_OK) m = make_tensor_map_bf16(&t[3], L.w_proj, d, F, 128);
+            m = make_map(&t[0], L.w_qkv, 3 * d, d, 128);
+            if (m == SSD_OK) m = make_map(&t[1], L.w_o, d, d, 128);
+            if (m == SSD_OK) m = make_map(&t[2], L.w_fc, F, d, 128);
+            if (m == SSD_OK) m = make_map(&t[3], L.w_proj, d, F, 128);
         }
         if (m != SSD_OK) return m;
         // LayerNorm-fold vectors of the cluster-reduced path, its statistics buffers, the timeline buffer
@@ -613,14 +665,9 @@ int ssd_w8_read(ssd_ctx *ctx, int32_t which, int32_t layer, uint8_t *codes_out, 
         const size_t rw[4] = {3 * d, d, F, d}, kw[4] = {d, d, d, F};
         codes = cw[which]; scales = sw[which]; rows = rw[which]; cols = kw[which];
     }
-    std::vector<uint8_t> tiled(w8_tiled_bytes(rows, cols)); // stored tile by tile; handed back row-major
-    CU(cudaMemcpyAsync(tiled.data(), codes, tiled.size(), cudaMemcpyDeviceToHost, ctx->stream));
+    CU(cudaMemcpyAsync(codes_out, codes, rows * cols, cudaMemcpyDeviceToHost, ctx->stream));
     CU(cudaMemcpyAsync(scales_out, scales, rows * sizeof(float), cudaMemcpyDeviceToHost, ctx->stream));
     CU(cudaStreamSynchronize(ctx->stream));
-    const size_t k_tiles = cols / 64;
-    for (size_t o = 0; o < rows; ++o)
-        for (size_t kt = 0; kt < k_tiles; ++kt)
-            memcpy(codes_out + o * cols + kt * 64, tiled.data() + ((o / 128) * k_tiles + kt) * 8192 + (o % 128) * 64, 64);
     return SSD_OK;
 }
 
@@ -899,6 +946,11 @@ int ssd_set_tuning(ssd_ctx *ctx, int32_t knob, int32_t value) {
     case SSD_TUNE_CLUSTER_REDUCE: if (value != 0 && value != 1) return SSD_ERR_BAD_ARG; ctx->use_cluster = value; break;
     case SSD_TUNE_ATTN_LOW_PLANE: if (value != 0 && value != 1) return SSD_ERR_BAD_ARG; ctx->attn_lo = value; break;
     case SSD_TUNE_HEAD_STATS: if (value != 0 && value != 1) return SSD_ERR_BAD_ARG; ctx->use_head_stats = value; ctx->head_logits = nullptr; break;
+    case SSD_TUNE_W8_PLANES:
+        if (!ctx->w8 || value < 2 || value > 4) return SSD_ERR_BAD_ARG;
+        ctx->w8_planes = value;
+        for (auto &am : ctx->act_maps) am.built = false; // (the maps' boxes hold that many planes)
+        break;
     case SSD_TUNE_CLUSTER_MAX: if (value < 1 || value > 16) return SSD_ERR_BAD_ARG; ctx->cl_max = value; break;
     case SSD_TUNE_CLUSTER_QKV: case SSD_TUNE_CLUSTER_O: case SSD_TUNE_CLUSTER_FC: case SSD_TUNE_CLUSTER_PROJ:
         if (value < 0 || value > 16) return SSD_ERR_BAD_ARG;

@@ -66,18 +66,19 @@ cudaError_t launch_tree_attention(const float *qkv, const StepInfo *info, size_t
 // `zero` may be null; if zero_from_info is set the zeroed buffer is info->logits instead.
 cudaError_t launch_ln_prep(const float *x, const float *g, const float *b, int n, int d, float eps, __nv_bfloat16 *a_hi, __nv_bfloat16 *a_lo,
                            float *zero, int zero_cols, const StepInfo *info, int zero_from_info, bool pdl, cudaStream_t s,
-                           unsigned long long *trace = nullptr);
+                           unsigned long long *trace = nullptr, uint8_t *planes8 = nullptr, size_t plane_stride = 0);
 cudaError_t launch_gelu_prep(const float *acc, int n, int F, __nv_bfloat16 *h_hi, __nv_bfloat16 *h_lo, bool pdl, cudaStream_t s,
-                             unsigned long long *trace = nullptr);
+                             unsigned long long *trace = nullptr, uint8_t *planes8 = nullptr, size_t plane_stride = 0);
+// (planes8, where a launcher takes it: instead of the bf16 planes write the four e4m3 planes [4][rows][K] the 8-bit projections
+//  read, plane_stride = rows * K bytes apart; see w8_planes.cuh)
 // (`trace`, where a launcher takes it: eight timestamp slots of this launch, see ptx::trace_mark; null = off)
 // Tensor maps are opaque 128-byte objects (CUtensorMap) built on the host.
 struct alignas(64) TensorMap { unsigned char bytes[128]; };
 int make_tensor_map_bf16(void *map_out, const void *base, uint64_t rows, uint64_t cols, uint32_t box_rows);
-// 8-bit weights: W[rows, cols] bf16 -> e4m3 codes and one power-of-two scale per row, the smallest that brings the row's
-// largest magnitude within the format's range (448); code = round-to-nearest-even(W / scale).  A row of zeros gets scale 1.
-// The codes are written tile by tile: code (o, k) at ((o / 128) * (cols / 64) + k / 64) * 8192 + (o % 128) * 64 + k % 64; the
-// buffer holds ceil(rows / 128) * (cols / 64) tiles and must be zeroed beforehand (rows past the matrix stay zero).
-size_t w8_tiled_bytes(size_t rows, size_t cols);
+int make_tensor_map_u8(void *map_out, const void *base, uint64_t rows, uint64_t cols, uint32_t box_rows);
+int make_tensor_map_u8_planes(void *map_out, const void *base, uint64_t rows, uint64_t cols, uint32_t box_rows, uint32_t box_planes);
+// 8-bit weights: W[rows, cols] bf16 -> e4m3 codes [rows, cols] and one power-of-two scale per row, the smallest that brings the
+// row's largest magnitude within the format's range (448); code = round-to-nearest-even(W / scale).  A row of zeros gets scale 1.
 cudaError_t launch_quantise_rows_e4m3(const void *w_bf16, size_t rows, size_t cols, uint8_t *codes, float *scales, cudaStream_t s);
 cudaError_t gemm_ws_prepare();
 cudaError_t prep_kernels_prepare();
@@ -87,13 +88,15 @@ cudaError_t prep_kernels_prepare();
 // half an SM's shared memory.
 // With `head` set the projection runs one CTA per output tile over the whole K (complete sums): plain stores, no clearing of Y
 // needed, and per (row, tile) the maximum, its lowest feature index and a non-finite flag at [row * n_tiles + tile].
-// With `w_codes` set the weights are 8-bit codes stored tile by tile (see launch_quantise_rows_e4m3), w_scale[out] their per-row
-// scales, and map_w is ignored.
+// With `w_scale` set the weights are 8-bit codes (map_w from make_tensor_map_u8, w_scale[out] their per-row scales) and the
+// activations e4m3 planes, the first w8_planes of the four (map_hi from make_tensor_map_u8_planes with that many planes per box;
+// map_lo unused); n <= 128 rows per launch, the rows
+// row0 .. row0 + n - 1 of the planes and of y; K need not be a multiple of 128; `head` is not supported.
 struct GemmHeadStats { float *val; int32_t *arg, *bad; };
 cudaError_t launch_gemm_ws(const void *map_w, const void *map_hi, const void *map_lo, float *y, const StepInfo *info, int ldy,
                            const float *bias, int n, int K, int out, int use_lo, int grid, int sm_count, int32_t *status, bool pdl,
                            cudaStream_t s, unsigned long long *trace = nullptr, const GemmHeadStats *head = nullptr,
-                           const float *w_scale = nullptr, const uint8_t *w_codes = nullptr);
+                           const float *w_scale = nullptr, int row0 = 0, int w8_planes = 4);
 // ---- projection with the split-K sums reduced inside a thread-block cluster (trees of up to 64 nodes) ----
 // What the epilogue does with the finished sums acc[i, o] (see k_gemm_cl.cu):
 enum { MODE_FOLD_STORE = 0, MODE_FOLD_GELU = 1, MODE_RESIDUAL = 2 };
@@ -138,7 +141,8 @@ size_t tree_attention_mma_smem(int n);
 cudaError_t tree_attention_mma_prepare();
 cudaError_t launch_tree_attention_mma(const float *qkv, const StepInfo *info, size_t layer_offset_elems, const TreeMeta &m, int n, int n_head,
                                       int cap, __nv_bfloat16 *o_hi, __nv_bfloat16 *o_lo, bool pdl, cudaStream_t s,
-                                      unsigned long long *trace = nullptr, bool lo_pairs = true);
+                                      unsigned long long *trace = nullptr, bool lo_pairs = true, uint8_t *planes8 = nullptr,
+                                      size_t plane_stride = 0);
 
 #define SSD_ACC_SUPPORT 1024
 struct AcceptScratch {

@@ -297,3 +297,23 @@ def test_w8_row_scale_rule_and_error_bound():
     assert np.array_equal(w8_oracle.dequantise_rows(q2, sc2), D)
     # and the grid values are bf16 numbers
     assert np.array_equal(ssd_synth.round_to_bf16(D), D)
+
+
+def test_four_e4m3_planes_carry_sixteen_bits():
+    """The operand format of the 8-bit projections, restated with the oracle's encoder: p0 = rn(x / 16), p1 = rn(x - 16 p0),
+    p2 = rn(16 r2), p3 = rn(256 r3) give x = 16 p0 + p1 + p2 / 16 + p3 / 256 to 2^-17 relative or 2^-18 absolute, whichever is
+    larger, for |x| up to 7168; three planes to 2^-13 / 2^-14; two to 2^-9 / 2^-10."""
+    from oracle import w8_oracle
+    val = w8_oracle.code_values()
+    rn = lambda a: val[w8_oracle.encode(a)]
+    rng = np.random.default_rng(3)
+    x = np.concatenate([rng.standard_normal(50000) * s for s in (1e-4, 1e-2, 1.0, 40.0, 2000.0)])
+    x = x[np.abs(x) <= 7168.0]
+    p0 = rn(x / 16); r1 = x - 16 * p0
+    p1 = rn(r1); r2 = r1 - p1
+    p2 = rn(16 * r2); r3 = r2 - p2 / 16
+    p3 = rn(256 * r3)
+    for planes, approx, rel, ab in ((4, 16 * p0 + p1 + p2 / 16 + p3 / 256, 2.0 ** -17, 2.0 ** -18),
+                                    (3, 16 * p0 + p1 + p2 / 16, 2.0 ** -13, 2.0 ** -14), (2, 16 * p0 + p1, 2.0 ** -9, 2.0 ** -10)):
+        err = np.abs(approx - x)
+        assert (err <= np.maximum(rel * np.abs(x), ab)).all(), planes
