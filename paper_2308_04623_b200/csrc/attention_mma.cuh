@@ -238,10 +238,15 @@ __device__ __forceinline__ void work_item(int tid, int bar_id, unsigned char *sm
         for (int m = 0; m < 2; ++m) {
             float c[4] = {0.f, 0.f, 0.f, 0.f}, cl[4] = {0.f, 0.f, 0.f, 0.f}; // q's high and low parts: two chains of four, not one of eight
             const uint4 k0 = cur.k[m][0], k1 = cur.k[m][1];
-            mma_bf16(c, qh[0], k0.x, k0.y); if (LO) mma_bf16(cl, ql[0], k0.x, k0.y);
-            mma_bf16(c, qh[1], k0.z, k0.w); if (LO) mma_bf16(cl, ql[1], k0.z, k0.w);
-            mma_bf16(c, qh[2], k1.x, k1.y); if (LO) mma_bf16(cl, ql[2], k1.x, k1.y);
-            mma_bf16(c, qh[3], k1.z, k1.w); if (LO) mma_bf16(cl, ql[3], k1.z, k1.w);
+            if (LO) {
+                mma_bf16(c, qh[0], k0.x, k0.y); mma_bf16(cl, ql[0], k0.x, k0.y);
+                mma_bf16(c, qh[1], k0.z, k0.w); mma_bf16(cl, ql[1], k0.z, k0.w);
+                mma_bf16(c, qh[2], k1.x, k1.y); mma_bf16(cl, ql[2], k1.x, k1.y);
+                mma_bf16(c, qh[3], k1.z, k1.w); mma_bf16(cl, ql[3], k1.z, k1.w);
+            } else { // (two chains of two: cl takes the second half of the dimensions)
+                mma_bf16(c, qh[0], k0.x, k0.y); mma_bf16(cl, qh[2], k1.x, k1.y);
+                mma_bf16(c, qh[1], k0.z, k0.w); mma_bf16(cl, qh[3], k1.z, k1.w);
+            }
 #pragma unroll
             for (int q = 0; q < 4; ++q) c[q] += cl[q];
 #pragma unroll
@@ -317,11 +322,11 @@ __device__ __forceinline__ void work_item(int tid, int bar_id, unsigned char *sm
         const int r = slot >> 4, c0 = (slot & 15) * 4, row = tile0 + r;
         if (row < n) {
             float M = -INFINITY;
-#pragma unroll 2
+#pragma unroll
             for (int w = 0; w < NW; ++w) M = fmaxf(M, s_merge[((size_t)w * 16 + r) * 66]);
             float L = 0.f, acc[4] = {0.f, 0.f, 0.f, 0.f};
-#pragma unroll 2
-            for (int w = 0; w < NW; ++w) {
+#pragma unroll
+            for (int w = 0; w < NW; ++w) { // (unrolled: the warps' partial results are fetched together, not one after the other)
                 const float *src = s_merge + ((size_t)w * 16 + r) * 66;
                 const float wgt = (src[0] == -INFINITY) ? 0.f : __expf(src[0] - M);
                 L += src[1] * wgt;
