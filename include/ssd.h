@@ -275,11 +275,14 @@ int ssd_kv_read(ssd_ctx *ctx, const ssd_kv *kv, int32_t layer, int32_t which, in
  *                                 acceptance 10 us faster.  0 = stream-K head adding partial sums at L2 into cleared logits
  *   SSD_TUNE_W8_PLANES [4]        SSD_DTYPE_BF16_W8 only: how many e4m3 planes of an activation the projections use, 2..4 (each carries
  *                                 4 significant bits; every plane less shortens the projections' epilogues)
+ *   SSD_TUNE_STAGE_KV_FROM [128]  bf16 models: trees of at least this many nodes get one more kernel per layer, which writes the tree's
+ *                                 K / V rows to the cache's scratch slots so that the attention reads every key block from the cache
+ *                                 (otherwise each 16-node tile of a head converts and stages the whole tree's keys itself); 0 = never
  *   SSD_TUNE_KERNEL_TRACE [0]     record a timeline of every kernel of a bf16 forward (see ssd_get_phase_trace)
  */
 enum { SSD_TUNE_LOW_PLANE = 0, SSD_TUNE_DEPENDENT_LAUNCH = 1, SSD_TUNE_GRAPH = 2, SSD_TUNE_GEMM_CTAS = 3, SSD_TUNE_CLUSTER_REDUCE = 4,
        SSD_TUNE_CLUSTER_MAX = 5, SSD_TUNE_ATTN_LOW_PLANE = 6, SSD_TUNE_HEAD_CTAS = 7, SSD_TUNE_KERNEL_TRACE = 8, SSD_TUNE_CLUSTER_QKV = 9, SSD_TUNE_CLUSTER_O = 10,
-       SSD_TUNE_CLUSTER_FC = 11, SSD_TUNE_CLUSTER_PROJ = 12, SSD_TUNE_HEAD_STATS = 13, SSD_TUNE_W8_PLANES = 14 };
+       SSD_TUNE_CLUSTER_FC = 11, SSD_TUNE_CLUSTER_PROJ = 12, SSD_TUNE_HEAD_STATS = 13, SSD_TUNE_W8_PLANES = 14, SSD_TUNE_STAGE_KV_FROM = 15 };
 int ssd_set_tuning(ssd_ctx *ctx, int32_t knob, int32_t value);
 
 /*

@@ -30,9 +30,9 @@ constexpr int KROW = DH + 8;     // shared-memory K row stride (elements): 144 B
 constexpr int MAX_SPLITS = 4;
 constexpr int QROW = DH + 4;     // shared-memory row stride (floats) of the 16 query rows
 
-__host__ __device__ inline size_t smem_bytes(int n, int NW = NW_MAX) {
-    // sized for the worst prefix alignment: up to 15 prefix-tail keys plus n tree keys
-    const int lk_pad = (n + 15 + 15) & ~15;
+__host__ __device__ inline size_t smem_bytes(int n, int NW = NW_MAX, bool staged = false) {
+    // sized for the worst prefix alignment: up to 15 prefix-tail keys plus n tree keys (none when the tree's rows are read from the cache)
+    const int lk_pad = staged ? 0 : (n + 15 + 15) & ~15;
     const int vrow = lk_pad + 8;
     return (size_t)lk_pad * KROW * 2 + (size_t)DH * vrow * 2 + (size_t)NW * 16 * 66 * 4 + (size_t)16 * QROW * 4 + 16 * SSD_ANC_WORDS * 8 + 16;
 }
@@ -78,14 +78,17 @@ struct BlockFrags {
 // first blocks (written by earlier steps) are requested first, then it waits for the kernel that produced `qkv`.
 // LO: q and the softmax weights enter the tensor cores as hi + lo pairs (two MMAs each); without it as one bf16 value, which
 // rounds them as coarsely as the cache already rounds K and V.
-template <int NW, bool PREFETCH, bool PDL_WAIT = false, bool LO = true>
+// STAGED: a kernel before this one has already written the tree's K / V rows (bf16) to the cache's scratch slots kv_len + i and zeroed
+// the rest of the last 16-key block: every block is read from the cache, nothing is staged in shared memory (large trees: with
+// sixteen 16-node tiles per head, sixteen CTAs would otherwise each convert and stage the whole tree's keys).
+template <int NW, bool PREFETCH, bool PDL_WAIT = false, bool LO = true, bool STAGED = false>
 __device__ __forceinline__ void work_item(int tid, int bar_id, unsigned char *smem_raw, int h, int tile0, int split, int n_splits,
                                           bool store_scratch, const float *__restrict__ qkv, const StepInfo *__restrict__ info,
                                           size_t layer_offset, const TreeMeta &meta, int n, int d, int cap, const Output &out,
                                           unsigned long long *trace = nullptr) {
     const int warp = tid >> 5, lane = tid & 31, g = lane >> 2, t = lane & 3;
     const int P = info->kv_len, Pf = P & ~15, n_keys = P + n;
-    const int local_keys = n_keys - Pf;             // keys held in shared memory: prefix tail + tree
+    const int local_keys = STAGED ? 0 : n_keys - Pf; // keys held in shared memory: prefix tail + tree
     const int lk_pad = (local_keys + 15) & ~15;
     const int vrow = lk_pad + 8;                    // shared V^T row stride (elements)
     __nv_bfloat16 *kc = reinterpret_cast<__nv_bfloat16 *>(info->kbase) + layer_offset + (size_t)h * cap * DH;  // [cap, 64]
@@ -98,7 +101,7 @@ __device__ __forceinline__ void work_item(int tid, int bar_id, unsigned char *sm
 
     const int n_blocks = (n_keys + 15) >> 4;
     const int b_lo = (n_blocks * split) / n_splits, b_hi = (n_blocks * (split + 1)) / n_splits;
-    const bool need_local = store_scratch || (b_hi << 4) > Pf;
+    const bool need_local = !STAGED && (store_scratch || (b_hi << 4) > Pf);
 
     // ---- first blocks' K/V fragments from the cache (global): they depend on no kernel of this step
     auto load_global = [&](int b, BlockFrags &f) {
@@ -122,6 +125,10 @@ __device__ __forceinline__ void work_item(int tid, int bar_id, unsigned char *sm
         }
 #pragma unroll
         for (int dt = 0; dt < 8; ++dt) f.v[dt] = *reinterpret_cast<const uint2 *>(s_v + (size_t)(8 * dt + g) * vrow + kb + 4 * t);
+    };
+    auto load_late = [&](int blk, BlockFrags &f) { // a block that holds rows of this step's tree
+        if (STAGED) load_global(blk, f);
+        else load_local(blk, f);
     };
     BlockFrags cur, nxt;
     int b = b_lo + warp;
@@ -223,12 +230,12 @@ __device__ __forceinline__ void work_item(int tid, int bar_id, unsigned char *sm
 #pragma unroll
         for (int q = 0; q < 4; ++q) oacc[dt][q] = 0.f;
 
-    if (b < b_hi && (b << 4) >= Pf) load_local(b, cur);
+    if (b < b_hi && (b << 4) >= Pf) load_late(b, cur);
     while (b < b_hi) {
         const int kb = b << 4, nb = b + NW;
         if (PREFETCH && nb < b_hi && !nxt_ready) { // fetch the next block while this one is computed
             if ((nb << 4) < Pf) load_global(nb, nxt);
-            else load_local(nb, nxt);
+            else load_late(nb, nxt);
         }
         nxt_ready = false;
         const bool tree_block = kb + 16 > P; // only such blocks need the ancestor mask
@@ -295,7 +302,7 @@ __device__ __forceinline__ void work_item(int tid, int bar_id, unsigned char *sm
             cur = nxt;
         } else if (b < b_hi) {
             if ((b << 4) < Pf) load_global(b, cur);
-            else load_local(b, cur);
+            else load_late(b, cur);
         }
     }
     // row sums over the four lanes of a quad

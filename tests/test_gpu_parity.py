@@ -12,6 +12,13 @@ TOL_F32 = 1e-4   # fp32 configuration (stated target)
 TOL_BF16 = 3e-2  # bf16 weights (stated target)
 
 
+def forward_launches(n_layer, n, w8=False):
+    """Kernels of one default-path bf16 forward: tree preparation, clearing of the logits, embedding; eight per layer - nine from 128
+    nodes on, where a kernel of its own writes the tree's K / V rows to the cache; final LayerNorm and LM head.  With 8-bit weights a
+    projection takes 128 nodes per launch, so larger trees run each of the 4 L + 1 projections twice."""
+    return 3 + (8 + (1 if n >= 128 else 0)) * n_layer + 2 + ((4 * n_layer + 1) if (w8 and n > 128) else 0)
+
+
 @pytest.fixture(scope="module")
 def ssd():
     import paper_2308_04623_b200 as m
@@ -574,7 +581,7 @@ def test_head_with_row_statistics_and_stream_k_head_give_the_same_logits(name, n
         p.ctx.set_tuning(ssd.SSD_TUNE_HEAD_STATS, 0)
         before = p.ctx.kernel_launches()
         plain, _, buf2 = p.verify(tokens, parent)
-        assert p.ctx.kernel_launches() - before == 3 + 8 * p.cfg["n_layer"] + 2
+        assert p.ctx.kernel_launches() - before == forward_launches(p.cfg["n_layer"], n)
         assert np.abs(plain - got).max() <= 1e-3 and np.abs(plain - want).max() <= TOL_BF16
         before = p.ctx.kernel_launches()
         opath, onxt, _ = ssd_oracle.accept_tree(plain.astype(np.float32), None, tokens, parent, mode=0)
@@ -769,7 +776,7 @@ def test_w8_logits_against_the_oracle_and_the_bf16_path(ssd, util, cfg_name):
         before = p8.ctx.kernel_launches()
         got8, want, buf8 = p8.verify(tok, par)
         # (a projection on the 8-bit tensor-core kind takes 128 nodes at most: larger trees run each one as two launches)
-        assert p8.ctx.kernel_launches() - before == (3 + 8 * L + 2 if n <= 128 else 3 + 12 * L + 3)
+        assert p8.ctx.kernel_launches() - before == forward_launches(L, n, w8=True)
         got16, _, _ = p16.verify(tok, par)
         assert np.isfinite(got8).all()
         assert np.abs(got8 - want).max() <= TOL_BF16, n
@@ -826,3 +833,33 @@ def test_w8_plane_count(ssd, util):
     with pytest.raises(ssd.SsdError):
         p16.ctx.set_tuning(ssd.SSD_TUNE_W8_PLANES, 3)
     p16.close()
+
+
+@pytest.mark.parametrize("prefix", [0, 5, 16, 37])
+def test_tree_rows_read_from_the_cache_give_the_same_logits(ssd, util, prefix):
+    """Large trees: a kernel of its own writes the tree's K / V rows to the cache's scratch slots (and zeroes the rest of the last
+    16-key block) and the attention reads every block from the cache.  Against the oracle and against the path in which every
+    node tile stages the tree's keys itself, for prefixes that end on and off a 16-key boundary, with commits in between (the
+    scratch rows then become committed ones); forcing the path on a small tree covers the case of a single partial block."""
+    rng = np.random.default_rng(61 + prefix)
+    p = util.Pair("ragged_bf16", seed=3, qk_gain=3.0)
+    V, L = p.V, p.cfg["n_layer"]
+    if prefix:
+        p.prefill(ssd_synth.uniform_tokens(prefix, V, rng))
+    for n in (70, 131, 256, 9):
+        par = ssd_synth.tree_random(n, 7, rng)
+        tok = ssd_synth.uniform_tokens(n, V, rng)
+        p.ctx.set_tuning(ssd.SSD_TUNE_STAGE_KV_FROM, 1)
+        before = p.ctx.kernel_launches()
+        got, want, _ = p.verify(tok, par)
+        assert p.ctx.kernel_launches() - before == 3 + 9 * L + 2
+        p.ctx.set_tuning(ssd.SSD_TUNE_STAGE_KV_FROM, 0)
+        before = p.ctx.kernel_launches()
+        plain, _, _ = p.verify(tok, par)
+        assert p.ctx.kernel_launches() - before == 3 + 8 * L + 2
+        assert np.abs(got - want).max() <= TOL_BF16, (prefix, n)
+        assert np.abs(got - plain).max() <= 1e-3, (prefix, n)
+        path = ssd_synth.path_to(par, int(rng.integers(0, n)))
+        p.commit(path)
+    assert p.ctx.device_status() == 0
+    p.close()
