@@ -397,12 +397,16 @@ def run_sweep(args, local, peaks):
     run.close()
     del run
     # ---- GPT-2-XL-shaped model: tree sizes 8..256, random parents with depth <= 8
-    run = Runner("gpt2_xl", 512, local, args.tune)
-    rows_xl = []
-    for n in (8, 16, 32, 64, 128, 256):
-        parent = ssd_synth.tree_random(n, 8, run.rng)
-        toks = [ssd_synth.uniform_tokens(n, run.V, run.rng) for _ in range(4)]
-        rows_xl.append(sweep_entry("gpt2_xl verify, random tree of depth <= 8", run.cfg, n, 512, run.time_steps(parent, toks, steps, warm), peaks))
+    # (one model, prefilled to the longest prefix; the shorter prefixes are the same cache rolled back)
+    run = Runner("gpt2_xl", 960, local, args.tune)
+    rows_xl, other_prefixes = [], []
+    trees = {n: (ssd_synth.tree_random(n, 8, run.rng), [ssd_synth.uniform_tokens(n, run.V, run.rng) for _ in range(4)]) for n in (8, 16, 32, 64, 128, 256)}
+    for P in (960, 512, 128):
+        run.kv.rollback(P)
+        run.P = P
+        for n, (parent, toks) in trees.items():
+            e = sweep_entry("gpt2_xl verify, random tree of depth <= 8", run.cfg, n, P, run.time_steps(parent, toks, steps if P == 512 else 10, warm), peaks)
+            (rows_xl if P == 512 else other_prefixes).append(e if P == 512 else {k: e[k] for k in ("n_nodes", "prefix", "verify_us", "frac_hbm_measured", "frac_tensor_sustained", "bound_us")})
     cfg = run.cfg
     run.close()
     del run
@@ -413,7 +417,7 @@ def run_sweep(args, local, peaks):
             cross = n
             break
     t = [r["verify_us"]["median"] for r in rows_xl]
-    out["config5"] = {"rows": rows_xl, "crossover_nodes_of_the_bounds": cross,
+    out["config5"] = {"rows": rows_xl, "rows_prefix_960_and_128": other_prefixes, "crossover_nodes_of_the_bounds": cross,
                       "measured_us_per_node_beyond_64": (t[5] - t[3]) / (256 - 64),
                       "note": "below the crossover the forward can at best run at the HBM bound, above it at the tensor bound; measured times "
                               "are several times either bound (a chain of dependent kernels), and grow roughly linearly in the tree size from 64 nodes on"}
