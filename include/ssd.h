@@ -106,7 +106,7 @@ typedef struct {
  * Create a context on CUDA device `device`, enqueueing on `cuda_stream` (a cudaStream_t passed
  * as void*; NULL = the legacy default stream).  Supported shapes: d_head = 64,
  * n_head * d_head = d_model, d_model and d_ff multiples of 64, 1 <= max_nodes <= 256,
- * n_ctx >= 2.  Allocates the device workspaces.  *out is NULL on failure.
+ * n_ctx >= 2; an fp32 model also needs n_ctx + max_nodes <= 3008 (its attention's shared memory).  Allocates the device workspaces.  *out is NULL on failure.
  */
 int ssd_create(const ssd_config *cfg, int device, void *cuda_stream, ssd_ctx **out);
 

@@ -149,6 +149,9 @@ __global__ void __launch_bounds__(WARPS * 32) tree_attention_kernel(const float 
 }
 } // namespace
 
+// Shared memory of one CTA for key lists of up to max_keys entries (it must fit the 48 KB a kernel gets without opting in to more).
+size_t tree_attention_smem(int max_keys) { return sizeof(float) * (WARPS * DH + (size_t)WARPS * max_keys); }
+
 cudaError_t launch_tree_attention(const float *qkv, const StepInfo *info, size_t layer_offset_elems, int dtype, const TreeMeta &m, int n,
                                   int max_keys, int n_head, int cap, float *o, __nv_bfloat16 *o_hi, __nv_bfloat16 *o_lo, bool pdl,
                                   cudaStream_t s) {
@@ -161,7 +164,7 @@ cudaError_t launch_tree_attention(const float *qkv, const StepInfo *info, size_t
     groups = (n + per - 1) / per;
     // shared memory is sized for the longest key list the cache allows, so that one captured
     // launch serves every prefix length
-    const size_t smem = sizeof(float) * (WARPS * DH + (size_t)WARPS * max_keys);
+    const size_t smem = tree_attention_smem(max_keys);
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3(n_head, groups);
     cfg.blockDim = dim3(WARPS * 32);

@@ -435,6 +435,8 @@ int ssd_create(const ssd_config *cfg, int device, void *cuda_stream, ssd_ctx **o
     if (cfg->d_head != 64 || cfg->n_head * cfg->d_head != cfg->d_model || cfg->d_model % 64 || cfg->d_ff % 64 ||
         cfg->max_nodes > SSD_MAX_NODES || cfg->d_model > 8192)
         return SSD_ERR_UNSUPPORTED;
+    // (the fp32 model's attention keeps one score per key and warp in shared memory)
+    if (cfg->dtype == SSD_DTYPE_F32 && tree_attention_smem(cfg->n_ctx + cfg->max_nodes) > 48 * 1024) return SSD_ERR_UNSUPPORTED;
     int count = 0;
     if (cudaGetDeviceCount(&count) != cudaSuccess || device < 0 || device >= count) return SSD_ERR_CUDA;
     ssd_ctx *ctx = new (std::nothrow) ssd_ctx();

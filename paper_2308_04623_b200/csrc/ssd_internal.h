@@ -57,6 +57,7 @@ cudaError_t launch_gemm_simple(const float *a, const void *W, int dtype, const f
                                float *y, cudaStream_t s);
 // Tree attention for one layer.  qkv: [n, 3d] fp32 (bias included).  kcache/vcache: this layer's
 // [H, cap, 64] rows (float or bf16).  Writes the nodes' K/V to slots kv_len + i and o[n, d].
+size_t tree_attention_smem(int max_keys);
 cudaError_t launch_tree_attention(const float *qkv, const StepInfo *info, size_t layer_offset_elems, int dtype, const TreeMeta &m, int n,
                                   int max_keys, int n_head, int cap, float *o, __nv_bfloat16 *o_hi, __nv_bfloat16 *o_lo, bool pdl,
                                   cudaStream_t s);

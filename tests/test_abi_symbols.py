@@ -48,6 +48,8 @@ def test_unsupported_shapes_are_refused_before_touching_a_device():
     assert lib.ssd_create(C.byref(bad_head), 0, None, C.byref(out)) == ssd.SSD_ERR_UNSUPPORTED
     too_many = ssd_config(2, 256, 4, 64, 1024, 1000, 128, 257, 0, 1e-5)
     assert lib.ssd_create(C.byref(too_many), 0, None, C.byref(out)) == ssd.SSD_ERR_UNSUPPORTED
+    long_fp32 = ssd_config(2, 256, 4, 64, 1024, 1000, 3000, 64, 0, 1e-5)   # fp32 attention: n_ctx + max_nodes above 3008 keys
+    assert lib.ssd_create(C.byref(long_fp32), 0, None, C.byref(out)) == ssd.SSD_ERR_UNSUPPORTED
     bad_dtype = ssd_config(2, 256, 4, 64, 1024, 1000, 128, 64, 7, 1e-5)
     assert lib.ssd_create(C.byref(bad_dtype), 0, None, C.byref(out)) == ssd.SSD_ERR_BAD_ARG
 
