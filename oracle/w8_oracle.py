@@ -55,16 +55,13 @@ def encode(x) -> np.ndarray:
 def row_scales(w) -> np.ndarray:
     """Per row: the smallest power of two s with max|w| <= 448 s; 1 for a row of zeros."""
     amax = np.max(np.abs(np.asarray(w, dtype=np.float64)), axis=1)
-    s = np.ones(len(amax), dtype=np.float64)
-    for i, a in enumerate(amax):
-        if a > 0.0:
-            e = int(np.ceil(np.log2(a / E4M3_MAX)))
-            while a > E4M3_MAX * 2.0 ** e:          # (guards the rounding of log2)
-                e += 1
-            while a <= E4M3_MAX * 2.0 ** (e - 1):
-                e -= 1
-            s[i] = 2.0 ** e
-    return s.astype(np.float32)
+    pos = amax > 0.0
+    a = np.where(pos, amax, 1.0)
+    e = np.ceil(np.log2(a / E4M3_MAX))
+    e = np.where(a > E4M3_MAX * 2.0 ** e, e + 1, e)            # (guards the rounding of log2, either way)
+    e = np.where(a <= E4M3_MAX * 2.0 ** (e - 1), e - 1, e)
+    assert np.all(a <= E4M3_MAX * 2.0 ** e) and np.all(a > E4M3_MAX * 2.0 ** (e - 1))
+    return np.where(pos, 2.0 ** e, 1.0).astype(np.float32)
 
 
 def quantise_rows(w):

@@ -15,10 +15,10 @@ pytestmark = pytest.mark.gpu
 TOL_BF16 = 3e-2
 
 
-def _run(name, P, trees, seed=0, chunk=256):
+def _run(name, P, trees, seed=0, chunk=256, **pair_args):
     from tests import gpu_util
     import paper_2308_04623_b200 as ssd
-    p = gpu_util.Pair(name, seed=seed)
+    p = gpu_util.Pair(name, seed=seed, **pair_args)
     worst = {}
     fragile = 0
     try:
@@ -75,3 +75,12 @@ def test_gpt2_xl_shape_random_trees():
         for n in (8, 128):
             yield "n=%d" % n, ssd_synth.uniform_tokens(n, p.V, rng), ssd_synth.tree_random(n, 8, rng)
     _run("gpt2_xl", 128, trees, chunk=128)
+
+
+def test_gpt2_large_shape_8bit_weights():
+    """The benchmark's shape with the streamed matrices as 8-bit codes (model on the code grid, so that the oracle holds the same
+    numbers): the 32-node tree bench.py times and a 160-node tree, which runs every projection as two launches."""
+    def trees(p, rng):
+        yield "n=32", ssd_synth.uniform_tokens(32, p.V, rng), ssd_synth.tree_branching(32, (4, 2, 2, 1, 1))
+        yield "n=160", ssd_synth.uniform_tokens(160, p.V, rng), ssd_synth.tree_random(160, 8, rng)
+    _run("gpt2_large", 256, trees, on_grid=True, dtype="bf16_w8")
