@@ -175,8 +175,8 @@ gemm_ws_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant_
     } else if (warp == 0) {
         // ===================== TMA producer =====================
         if (lane == 0 && u1 > u0) {
-            ptx::prefetch_tensormap(&map_hi);
-            if (!W8 && p.use_lo) ptx::prefetch_tensormap(&map_lo);
+            if (W8 || !p.use_lo) ptx::prefetch_tensormap(&map_hi);
+            else ptx::prefetch_tensormap(&map_lo);
             const uint64_t pol = ptx::policy_evict_first();
             const uint32_t tx = (uint32_t)stage_bytes;
             // (phase 1, the weight tiles of the first `pre` units, was issued before the CTA-wide set-up barrier)
@@ -199,8 +199,10 @@ gemm_ws_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant_
                 if (W8) {
                     ptx::tma_load_3d(st + A_BYTES, &map_hi, kt * KT, p.row0, 0, &bars->full[s]);
                 } else {
-                    ptx::tma_load_2d(st + A_BYTES, &map_hi, kt * TILE_K, 0, &bars->full[s]);
-                    if (p.use_lo) ptx::tma_load_2d(st + A_BYTES + b_bytes, &map_lo, kt * TILE_K, 0, &bars->full[s]);
+                    // (with the lo plane: ONE box over both planes - they are adjacent in memory as in the stage - since every copy
+                    //  this one thread issues costs it some 50-100 ns ahead of the first MMA)
+                    if (p.use_lo) ptx::tma_load_3d(st + A_BYTES, &map_lo, kt * TILE_K, 0, 0, &bars->full[s]);
+                    else ptx::tma_load_2d(st + A_BYTES, &map_hi, kt * TILE_K, 0, &bars->full[s]);
                 }
                 if (bars->abort) ok = false;
                 if (++kt == p.k_tiles) { kt = 0; ++tile; }
@@ -437,6 +439,20 @@ int make_tensor_map_u8_planes(void *map_out, const void *base, uint64_t rows, ui
     cuuint32_t box[3] = {2 * TILE_K, box_rows, box_planes};
     cuuint32_t estr[3] = {1, 1, 1};
     CUresult r = fn((CUtensorMap *)map_out, CU_TENSOR_MAP_DATA_TYPE_UINT8, 3, const_cast<void *>(base), dims, strides, box, estr,
+                    CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                    CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    return r == CUDA_SUCCESS ? SSD_OK : SSD_ERR_CUDA;
+}
+
+// The bf16 hi and lo planes of an activation buffer, adjacent in memory ([2][rows][cols]): ONE box takes [2][box_rows][64].
+int make_tensor_map_bf16_pair(void *map_out, const void *base, uint64_t rows, uint64_t cols, uint32_t box_rows) {
+    EncodeTiledFn fn = encode_fn();
+    if (!fn) return SSD_ERR_CUDA;
+    cuuint64_t dims[3] = {cols, rows, 2};
+    cuuint64_t strides[2] = {cols * 2, rows * cols * 2};
+    cuuint32_t box[3] = {TILE_K, box_rows, 2};
+    cuuint32_t estr[3] = {1, 1, 1};
+    CUresult r = fn((CUtensorMap *)map_out, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void *>(base), dims, strides, box, estr,
                     CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
                     CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
     return r == CUDA_SUCCESS ? SSD_OK : SSD_ERR_CUDA;

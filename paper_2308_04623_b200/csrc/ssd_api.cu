@@ -36,7 +36,7 @@ struct ssd_ctx {
     __nv_bfloat16 *a_hi, *a_lo, *o_hi, *o_lo, *h_hi, *h_lo;
     // activation planes as tensor maps whose box is the whole padded batch [n_pad rows x 64]: one TMA operation per
     // plane and k tile (index n_pad / 16 - 1; built on first use)
-    struct ActMaps { TensorMap a_hi, a_lo, o_hi, o_lo, h_hi, h_lo; bool built; };
+    struct ActMaps { TensorMap a_hi, a_lo, o_hi, o_lo, h_hi, h_lo, a_pair, o_pair, h_pair; bool built; }; // (_pair: hi and lo planes as one box)
     ActMaps act_maps[SSD_MAX_NODES / 16];
     size_t plane_rows;
     TensorMap map_wte;
@@ -185,6 +185,9 @@ static const ssd_ctx::ActMaps *act_maps_pad(ssd_ctx *ctx, int n_pad) {
         if (m == SSD_OK) m = make_tensor_map_bf16(&am.o_lo, ctx->o_lo, rows, d, n_pad);
         if (m == SSD_OK) m = make_tensor_map_bf16(&am.h_hi, ctx->h_hi, rows, F, n_pad);
         if (m == SSD_OK) m = make_tensor_map_bf16(&am.h_lo, ctx->h_lo, rows, F, n_pad);
+        if (m == SSD_OK) m = make_tensor_map_bf16_pair(&am.a_pair, ctx->a_hi, rows, d, n_pad);
+        if (m == SSD_OK) m = make_tensor_map_bf16_pair(&am.o_pair, ctx->o_hi, rows, d, n_pad);
+        if (m == SSD_OK) m = make_tensor_map_bf16_pair(&am.h_pair, ctx->h_hi, rows, F, n_pad);
         if (m != SSD_OK) return nullptr;
         am.built = true;
     }
@@ -271,7 +274,7 @@ cudaError_t enqueue_forward(ssd_ctx *ctx, int n, int cap, const NodeList &tk, co
         }
         const int hgrid = head_grid_for(ctx, n);
         Q(launch_ln_prep(ctx->x, ctx->lnf_g, ctx->lnf_b, n, d, c.ln_eps, ctx->a_hi, a_lo, nullptr, 0, info, 0, pdl, s, trace_slot(ctx, *kernels)));
-        Q(launch_gemm_ws(&ctx->map_wte, &amh->a_hi, &amh->a_lo, nullptr, info, c.vocab, nullptr, n, d, c.vocab, lo, hgrid, sms, ctx->d_status, pdl, s, trace_slot(ctx, *kernels), head));
+        Q(launch_gemm_ws(&ctx->map_wte, &amh->a_hi, &amh->a_pair, nullptr, info, c.vocab, nullptr, n, d, c.vocab, lo, hgrid, sms, ctx->d_status, pdl, s, trace_slot(ctx, *kernels), head));
         ctx->trace_count = ctx->trace_kernels ? 8 * *kernels : 0;
         return cudaSuccess;
     }
@@ -324,17 +327,17 @@ cudaError_t enqueue_forward(ssd_ctx *ctx, int n, int cap, const NodeList &tk, co
             const LayerWeights &L = ctx->layers[l];
             const TensorMap *t = &ctx->map_layers[(size_t)4 * l];
             Q(launch_ln_prep(ctx->x, L.ln1_g, L.ln1_b, n, d, c.ln_eps, ctx->a_hi, a_lo, ctx->qkv, 3 * d, info, 0, pdl, s, trace_slot(ctx, *kernels)));
-            Q(launch_gemm_ws(&t[0], &am->a_hi, &am->a_lo, ctx->qkv, info, 3 * d, L.b_qkv, n, d, 3 * d, lo, grid, sms, ctx->d_status, pdl, s, trace_slot(ctx, *kernels)));
+            Q(launch_gemm_ws(&t[0], &am->a_hi, &am->a_pair, ctx->qkv, info, 3 * d, L.b_qkv, n, d, 3 * d, lo, grid, sms, ctx->d_status, pdl, s, trace_slot(ctx, *kernels)));
             if (staged) Q(launch_kv_stage(ctx->qkv, info, l * layer_elems, n, c.n_head, cap, pdl, s, trace_slot(ctx, *kernels)));
             Q(launch_tree_attention_mma(ctx->qkv, info, l * layer_elems, ctx->meta, n, c.n_head, cap, ctx->o_hi, o_lo, pdl, s, trace_slot(ctx, *kernels), ctx->attn_lo != 0, nullptr, 0, staged));
-            Q(launch_gemm_ws(&t[1], &am->o_hi, &am->o_lo, ctx->x, info, d, L.b_o, n, d, d, lo, grid, sms, ctx->d_status, pdl, s, trace_slot(ctx, *kernels)));
+            Q(launch_gemm_ws(&t[1], &am->o_hi, &am->o_pair, ctx->x, info, d, L.b_o, n, d, d, lo, grid, sms, ctx->d_status, pdl, s, trace_slot(ctx, *kernels)));
             Q(launch_ln_prep(ctx->x, L.ln2_g, L.ln2_b, n, d, c.ln_eps, ctx->a_hi, a_lo, ctx->h, F, info, 0, pdl, s, trace_slot(ctx, *kernels)));
-            Q(launch_gemm_ws(&t[2], &am->a_hi, &am->a_lo, ctx->h, info, F, L.b_fc, n, d, F, lo, grid, sms, ctx->d_status, pdl, s, trace_slot(ctx, *kernels)));
+            Q(launch_gemm_ws(&t[2], &am->a_hi, &am->a_pair, ctx->h, info, F, L.b_fc, n, d, F, lo, grid, sms, ctx->d_status, pdl, s, trace_slot(ctx, *kernels)));
             Q(launch_gelu_prep(ctx->h, n, F, ctx->h_hi, h_lo, pdl, s, trace_slot(ctx, *kernels)));
-            Q(launch_gemm_ws(&t[3], &am->h_hi, &am->h_lo, ctx->x, info, d, L.b_proj, n, F, d, lo, grid, sms, ctx->d_status, pdl, s, trace_slot(ctx, *kernels)));
+            Q(launch_gemm_ws(&t[3], &am->h_hi, &am->h_pair, ctx->x, info, d, L.b_proj, n, F, d, lo, grid, sms, ctx->d_status, pdl, s, trace_slot(ctx, *kernels)));
         }
         Q(launch_ln_prep(ctx->x, ctx->lnf_g, ctx->lnf_b, n, d, c.ln_eps, ctx->a_hi, a_lo, nullptr, 0, info, 0, pdl, s, trace_slot(ctx, *kernels)));
-        Q(launch_gemm_ws(&ctx->map_wte, &am->a_hi, &am->a_lo, nullptr, info, c.vocab, nullptr, n, d, c.vocab, lo, hgrid, sms, ctx->d_status, pdl, s, trace_slot(ctx, *kernels), head));
+        Q(launch_gemm_ws(&ctx->map_wte, &am->a_hi, &am->a_pair, nullptr, info, c.vocab, nullptr, n, d, c.vocab, lo, hgrid, sms, ctx->d_status, pdl, s, trace_slot(ctx, *kernels), head));
         ctx->trace_count = ctx->trace_kernels ? 8 * *kernels : 0;
     } else {
         for (int l = 0; l < c.n_layer; ++l) {
@@ -496,8 +499,9 @@ int ssd_create(const ssd_config *cfg, int device, void *cuda_stream, ssd_ctx **o
     ctx->a_hi = ctx->a_lo = ctx->o_hi = ctx->o_lo = ctx->h_hi = ctx->h_lo = nullptr;
     if (ctx->tensor_path) {
         const size_t rows = n <= 32 ? 32 : ((n + 15) & ~size_t(15)); // operand planes hold whole 16-row boxes, at least two
-        A(&ctx->a_hi, rows * d); A(&ctx->a_lo, rows * d); A(&ctx->o_hi, rows * d); A(&ctx->o_lo, rows * d);
-        A(&ctx->h_hi, rows * (size_t)cfg->d_ff); A(&ctx->h_lo, rows * (size_t)cfg->d_ff);
+        // (a buffer's lo plane follows its hi plane, so that one 3-D copy fetches both)
+        A(&ctx->a_hi, 2 * rows * d); A(&ctx->o_hi, 2 * rows * d); A(&ctx->h_hi, 2 * rows * (size_t)cfg->d_ff);
+        if (rc == SSD_OK) { ctx->a_lo = ctx->a_hi + rows * d; ctx->o_lo = ctx->o_hi + rows * d; ctx->h_lo = ctx->h_hi + rows * (size_t)cfg->d_ff; }
         ctx->a8 = ctx->o8 = ctx->h8 = nullptr;
         if (ctx->w8) { A(&ctx->a8, 4 * rows * d); A(&ctx->o8, 4 * rows * d); A(&ctx->h8, 4 * rows * (size_t)cfg->d_ff); }
         ctx->head_tiles = (cfg->vocab + 127) / 128;

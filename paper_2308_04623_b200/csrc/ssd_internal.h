@@ -76,6 +76,7 @@ cudaError_t launch_gelu_prep(const float *acc, int n, int F, __nv_bfloat16 *h_hi
 // Tensor maps are opaque 128-byte objects (CUtensorMap) built on the host.
 struct alignas(64) TensorMap { unsigned char bytes[128]; };
 int make_tensor_map_bf16(void *map_out, const void *base, uint64_t rows, uint64_t cols, uint32_t box_rows);
+int make_tensor_map_bf16_pair(void *map_out, const void *base, uint64_t rows, uint64_t cols, uint32_t box_rows);
 int make_tensor_map_u8(void *map_out, const void *base, uint64_t rows, uint64_t cols, uint32_t box_rows);
 int make_tensor_map_u8_planes(void *map_out, const void *base, uint64_t rows, uint64_t cols, uint32_t box_rows, uint32_t box_planes);
 // 8-bit weights: W[rows, cols] bf16 -> e4m3 codes [rows, cols] and one power-of-two scale per row, the smallest that brings the
@@ -83,8 +84,9 @@ int make_tensor_map_u8_planes(void *map_out, const void *base, uint64_t rows, ui
 cudaError_t launch_quantise_rows_e4m3(const void *w_bf16, size_t rows, size_t cols, uint8_t *codes, float *scales, cudaStream_t s);
 cudaError_t gemm_ws_prepare();
 cudaError_t prep_kernels_prepare();
-// y[n, ldy] += X[n, K] . W[out, K]^T (+ bias once).  map_w: weights [out, K], boxes of 128 rows; map_hi / map_lo:
-// activation planes [rows >= n_pad, K], ONE box of n_pad rows (map_lo may be null when use_lo = 0).
+// y[n, ldy] += X[n, K] . W[out, K]^T (+ bias once).  map_w: weights [out, K], boxes of 128 rows; map_hi: the activations' hi plane
+// [rows >= n_pad, K], ONE box of n_pad rows; map_lo: with use_lo, the hi AND lo planes as one 3-D map (make_tensor_map_bf16_pair:
+// the lo plane follows the hi plane in memory), one box of [2][n_pad][64]; may be null when use_lo = 0.
 // If y is null the destination is info->logits.  `grid` CTAs share the units; with grid > sm_count each takes at most
 // half an SM's shared memory.
 // With `head` set the projection runs one CTA per output tile over the whole K (complete sums): plain stores, no clearing of Y
