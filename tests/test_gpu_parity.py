@@ -757,15 +757,16 @@ def test_w8_device_encoding_matches_the_oracle_encoding(ssd):
     ctx.close()
 
 
-@pytest.mark.parametrize("cfg_name", ["ragged_bf16", "tiny_bf16"])
-def test_w8_logits_against_the_oracle_and_the_bf16_path(ssd, util, cfg_name):
+@pytest.mark.parametrize("cfg_name,qk_gain", [("ragged_bf16", 1.0), ("tiny_bf16", 1.0), ("tiny_bf16", 4.0)])
+def test_w8_logits_against_the_oracle_and_the_bf16_path(ssd, util, cfg_name, qk_gain):
     """The model on the code grid held three ways - by the oracle (fp64), by the library as bf16 and by the library as 8-bit
     codes: 8-bit against the oracle within the bf16 tolerance over trees that span the single- and two-instruction operand
     layouts and ragged tails, with commits in between; 8-bit against bf16 to summation-order noise (same numbers, same
     products; only the order of the fp32 additions differs); same number of launches."""
     rng = np.random.default_rng(31)
-    p8 = util.Pair(cfg_name, seed=4, on_grid=True, dtype="bf16_w8")
-    p16 = util.Pair(cfg_name, seed=4, on_grid=True)
+    # (qk_gain > 1: sharpened attention, so that a wrong key, mask or plane shows in the logits)
+    p8 = util.Pair(cfg_name, seed=4, qk_gain=qk_gain, on_grid=True, dtype="bf16_w8")
+    p16 = util.Pair(cfg_name, seed=4, qk_gain=qk_gain, on_grid=True)
     V = p8.V
     prefix = ssd_synth.uniform_tokens(70, V, rng)
     p8.prefill(prefix); p16.prefill(prefix)
@@ -780,7 +781,8 @@ def test_w8_logits_against_the_oracle_and_the_bf16_path(ssd, util, cfg_name):
         got16, _, _ = p16.verify(tok, par)
         assert np.isfinite(got8).all()
         assert np.abs(got8 - want).max() <= TOL_BF16, n
-        assert np.abs(got8 - got16).max() <= 1e-3, n
+        # (sharpened attention magnifies a last-bit difference that moves a K / V value across a bf16 rounding boundary of the cache)
+        assert np.abs(got8 - got16).max() <= (1e-3 if qk_gain == 1.0 else 5e-3), n
         path, nxt = p8.ctx.accept_tree(buf8.data_ptr(), None, tok, par)
         opath, onext, margin = ssd_oracle.accept_tree(want.astype(np.float32), None, tok, par)
         if margin > 4 * TOL_BF16:
