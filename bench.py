@@ -78,8 +78,15 @@ class ClockSampler:
         except Exception:
             self.proc = None
 
+    def count(self) -> int:
+        try:
+            return sum(1 for line in open(self.path) if line.count(",") >= 6)
+        except Exception:
+            return 0
+
     def stop(self) -> dict:
-        out = {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "samples": 0}
+        out = {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "samples": 0,
+               "window": "warm-up steps, the timed region and identical untimed steps after it (the timed region alone is shorter than one sampling period)"}
         if not self.proc:
             return out
         time.sleep(0.15)
@@ -565,13 +572,17 @@ def run_gpu(args):
             dist.barrier()
         torch.cuda.synchronize()
 
-    run.time_steps(parent, token_sets, 1, args.warmup, draft, sampling)  # warm-up
     sampler = ClockSampler(local)
     if rank == 0:
         sampler.start()
+    run.time_steps(parent, token_sets, 1, args.warmup, draft, sampling)  # warm-up
     barrier()
     res = run.time_steps(parent, token_sets, args.steps, 0, draft, sampling)  # ---- the timed region: exactly K steps
     barrier()
+    if rank == 0:  # the same steps, untimed, until the sampler has seen the GPU under this load a few times
+        t_end = time.perf_counter() + 2.0
+        while sampler.proc and sampler.count() < 4 and time.perf_counter() < t_end:
+            run.time_steps(parent, token_sets, 20, 0, draft, sampling)
     clocks = sampler.stop() if rank == 0 else {}
     status = run.ctx.device_status()
     v = percentiles(res["verify_us"])
