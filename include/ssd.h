@@ -215,9 +215,10 @@ int ssd_accept_tree_noalloc(int device, void *cuda_stream, const float *logits, 
 /*
  * ssd_accept_tree with the proposal rows given as short index / value lists instead of dense rows: row c is zero except
  * row c[row_idx[c][e]] = row_val[c][e], e < entries (host arrays [n_nodes][entries], entries <= 1024; an index < 0 marks an
- * unused slot).  A deterministic proposal ("the second or third most likely tokens", Section 3.1) is a one-entry row with
- * value 1, a trigram row has four entries.  The rows are expanded on the device and the walk of ssd_accept_tree runs on
- * them: same rule, same results, same errors.
+ * unused slot; the indices of a row are distinct).  A deterministic proposal ("the second or third most likely tokens",
+ * Section 3.1) is a one-entry row with value 1, a trigram row has four entries.  Same rule, same results, same errors as
+ * ssd_accept_tree on the dense rows; the kernels read the lists themselves, and a refusal - which changes the residual law
+ * at the listed entries only - costs them O(entries) instead of two passes over the vocabulary.
  */
 int ssd_accept_tree_sparse(ssd_ctx *ctx, const float *logits, const int32_t *row_idx, const float *row_val, int32_t entries,
                            const int32_t *tokens, const int32_t *parent_idx, int32_t n_nodes, const ssd_sampling *sampling, ssd_rng *rng_state,

@@ -311,23 +311,51 @@ __device__ void draw_from(const double *__restrict__ r, int V, double u, int32_t
 // value in every thread), or -1 after ONE thread has written the extra token, drawn from r by inverse CDF, to *token_out.
 // The outcome depends on cur's own logits, its children's proposal rows and the counter-based uniforms only - not on how
 // the walk reached cur - so all nodes can be decided side by side.
-__device__ int node_decide(double *__restrict__ r, int cnt, const int32_t *__restrict__ sup, const float *__restrict__ draft,
+//
+// Proposal rows come dense (draft[c, :]) or as short lists (sp.idx / sp.val, [n][sp.entries], distinct indices, < 0 = unused).
+// With lists and a dense law a refusal touches the listed entries only: the residual max(0, r - q) differs from r there and
+// nowhere else, so r is kept UNNORMALISED with its total `norm` beside it (r_true = r / norm: the test u q[x] < r_true[x] becomes
+// u q[x] norm < r[x], the subtraction r - q norm, the new total norm minus what the listed entries lost) - O(entries) per refusal
+// instead of two passes over the vocabulary.  The extra token's inverse CDF sums r itself, so it needs no total.
+struct SparseRows { const int32_t *idx; const float *val; int entries; };
+__device__ __forceinline__ float q_at(const float *__restrict__ draft, const SparseRows &sp, int c, int V, int v) {
+    if (!sp.idx) return draft[(size_t)c * V + v];
+    for (int e = 0; e < sp.entries; ++e)
+        if (sp.idx[(size_t)c * sp.entries + e] == v) return sp.val[(size_t)c * sp.entries + e];
+    return 0.f;
+}
+__device__ int node_decide(double *__restrict__ r, int cnt, const int32_t *__restrict__ sup, const float *__restrict__ draft, const SparseRows sp,
                            const NodeList &tokens, const NodeList &parent, int n, int V, uint64_t seed, uint64_t step, int cur,
                            int32_t *__restrict__ token_out, BlockScratch &s) {
     const int tid = threadIdx.x;
+    double norm = 1.0; // total of r (lists with a dense law; every other case renormalises r in place and keeps 1)
     for (int c = cur + 1; c < n; ++c) {
         if (parent.v[c] != cur) continue;
-        const float *q = draft + (size_t)c * V;
+        const float *q = draft ? draft + (size_t)c * V : nullptr;
         const int x = tokens.v[c];
         const double u = uniform24(seed, step, 2u * (uint32_t)c);
-        if (u * (double)q[x] < r[x]) return c; // every thread evaluates the same test on the same values
+        if (u * (double)q_at(draft, sp, c, V, x) * norm < r[x]) return c; // every thread evaluates the same test on the same values
         // refusal: r <- max(0, r - q) renormalised (unchanged if nothing is left)
         __syncthreads(); // all threads have read r[x] before anyone rewrites it
         if (cnt >= 0) { // one support entry per thread
             const int iv = tid < cnt ? sup[tid] : 0;
-            const double val = tid < cnt ? fmax(r[iv] - (double)q[iv], 0.0) : 0.0;
+            const double val = tid < cnt ? fmax(r[iv] - (double)q_at(draft, sp, c, V, iv), 0.0) : 0.0;
             const double Z = block_sum(val, s);
             if (Z > 0.0 && tid < cnt) r[iv] = val / Z;
+        } else if (sp.idx) { // listed entries only
+            double lost = 0.0;
+            for (int e = tid; e < sp.entries; e += ACC_THREADS) {
+                const int v = sp.idx[(size_t)c * sp.entries + e];
+                if (v >= 0 && v < V) lost += r[v] - fmax(r[v] - (double)sp.val[(size_t)c * sp.entries + e] * norm, 0.0);
+            }
+            const double left = norm - block_sum(lost, s);
+            if (left > 0.0) {
+                for (int e = tid; e < sp.entries; e += ACC_THREADS) {
+                    const int v = sp.idx[(size_t)c * sp.entries + e];
+                    if (v >= 0 && v < V) r[v] = fmax(r[v] - (double)sp.val[(size_t)c * sp.entries + e] * norm, 0.0);
+                }
+                norm = left;
+            }
         } else {
             double zs = 0.0;
             for (int v = tid; v < V; v += ACC_THREADS) zs += fmax(r[v] - (double)q[v], 0.0);
@@ -379,7 +407,7 @@ __global__ void __launch_bounds__(ACC_THREADS) sample_walk_kernel(const float *_
             if (tid == 0) { result[0] = 1; result[1] = -1; result[2] = SSD_ERR_BAD_ARG; }
             return;
         }
-        const int c = node_decide(r, -1, nullptr, draft, tokens, parent, n, V, seed, step, cur, result + 1, s);
+        const int c = node_decide(r, -1, nullptr, draft, SparseRows{nullptr, nullptr, 0}, tokens, parent, n, V, seed, step, cur, result + 1, s);
         if (c < 0) {
             if (tid == 0) { result[0] = np; result[2] = SSD_OK; }
             return;
@@ -393,7 +421,7 @@ __global__ void __launch_bounds__(ACC_THREADS) sample_walk_kernel(const float *_
 
 // One CTA per node, after row_law_kernel: next[p] = the child accepted at p, -1 if none (bonus[p] then holds the extra
 // token), -2 if p's logits are unusable.
-__global__ void __launch_bounds__(ACC_THREADS) node_decide_kernel(const float *__restrict__ draft, NodeList tokens, NodeList parent, int n, int V,
+__global__ void __launch_bounds__(ACC_THREADS) node_decide_kernel(const float *__restrict__ draft, SparseRows sp, NodeList tokens, NodeList parent, int n, int V,
                                                                   uint64_t seed, uint64_t step, double *__restrict__ rows,
                                                                   const int32_t *__restrict__ row_bad, const int32_t *__restrict__ sup_idx,
                                                                   const int32_t *__restrict__ sup_cnt, int32_t *__restrict__ next,
@@ -405,7 +433,7 @@ __global__ void __launch_bounds__(ACC_THREADS) node_decide_kernel(const float *_
         return;
     }
     const int cnt = sup_cnt ? sup_cnt[p] : -1;
-    const int c = node_decide(rows + (size_t)p * V, cnt, cnt >= 0 ? sup_idx + (size_t)p * SSD_ACC_SUPPORT : nullptr, draft, tokens, parent, n, V,
+    const int c = node_decide(rows + (size_t)p * V, cnt, cnt >= 0 ? sup_idx + (size_t)p * SSD_ACC_SUPPORT : nullptr, draft, sp, tokens, parent, n, V,
                               seed, step, p, bonus + p, s);
     if (threadIdx.x == 0) next[p] = c;
 }
@@ -446,7 +474,8 @@ cudaError_t launch_accept(const float *logits, const float *draft_probs, const N
             // every node is decided by a CTA of its own (its law, then its children in order), then a walk follows the decisions
             int32_t *next = sc.row_arg, *bonus = sc.row_arg + n; // (row_arg holds 4 ints per node on this path)
             row_law_kernel<<<n, ACC_THREADS, 0, s>>>(logits, vocab, (double)temperature, top_k, rows, sc.row_bad, sc.sup_idx, sc.sup_cnt);
-            node_decide_kernel<<<n, ACC_THREADS, 0, s>>>(draft_probs, tokens, parent, n, vocab, seed, step, rows, sc.row_bad, sc.sup_idx, sc.sup_cnt,
+            const SparseRows sp = {sc.sp_idx, sc.sp_val, sc.sp_entries}; // (lists instead of dense rows: draft_probs is then not read)
+            node_decide_kernel<<<n, ACC_THREADS, 0, s>>>(draft_probs, sp, tokens, parent, n, vocab, seed, step, rows, sc.row_bad, sc.sup_idx, sc.sup_cnt,
                                                          next, bonus);
             chain_walk_kernel<<<1, 32, 0, s>>>(next, bonus, n, sc.result, sc.dev_status);
             *launches += 3;
@@ -591,6 +620,7 @@ cudaError_t noalloc_setup(int device, AcceptScratch *out) {
         slot.sc.result = (int32_t *)res;
         slot.sc.dev_status = nullptr;
         slot.sc.head_parts = 0;
+        slot.sc.sp_idx = nullptr; slot.sc.sp_val = nullptr; slot.sc.sp_entries = 0;
         slot.ready = true;
     }
     *out = slot.sc;

@@ -474,6 +474,7 @@ int ssd_create(const ssd_config *cfg, int device, void *cuda_stream, ssd_ctx **o
     ctx->acc.arg_parts = 4;
     ctx->acc.dev_status = nullptr;
     ctx->acc.head_parts = 0;
+    ctx->acc.sp_idx = nullptr; ctx->acc.sp_val = nullptr; ctx->acc.sp_entries = 0;
     ctx->head_val = nullptr; ctx->head_arg = ctx->head_bad = nullptr; ctx->head_tiles = 0; ctx->use_head_stats = 0;
     ctx->head_logits = nullptr; ctx->head_n = 0;
     A(&ctx->acc.r, (size_t)cfg->vocab); A(&ctx->acc.row_val, 4 * n); A(&ctx->acc.row_arg, 4 * n); A(&ctx->acc.row_bad, 4 * n); A(&ctx->acc.result, n + 4);
@@ -782,13 +783,15 @@ int ssd_verify_tree(ssd_ctx *ctx, const int32_t *tokens, const int32_t *parent_i
     return SSD_OK;
 }
 
-int ssd_accept_tree(ssd_ctx *ctx, const float *logits, const float *draft_probs, const int32_t *tokens, const int32_t *parent_idx,
-                    int32_t n_nodes, const ssd_sampling *sampling, ssd_rng *rng_state, int32_t *path_out, int32_t *n_path_out,
-                    int32_t *next_token_out) {
+namespace {
+// ssd_accept_tree, with the proposal rows dense (draft_probs) or as device lists (sp_idx / sp_val, [n][sp_entries]).
+int accept_impl(ssd_ctx *ctx, const float *logits, const float *draft_probs, const int32_t *sp_idx, const float *sp_val, int sp_entries,
+                const int32_t *tokens, const int32_t *parent_idx, int32_t n_nodes, const ssd_sampling *sampling, ssd_rng *rng_state,
+                int32_t *path_out, int32_t *n_path_out, int32_t *next_token_out) {
     if (!ctx || !logits || !tokens || !parent_idx || !sampling || !rng_state || !path_out || !n_path_out || !next_token_out)
         return SSD_ERR_BAD_ARG;
     if (sampling->mode != SSD_GREEDY && sampling->mode != SSD_SAMPLING) return SSD_ERR_BAD_ARG;
-    if (sampling->mode == SSD_SAMPLING && (!draft_probs || !(sampling->temperature > 0.f) || sampling->top_k < 0)) return SSD_ERR_BAD_ARG;
+    if (sampling->mode == SSD_SAMPLING && ((!draft_probs && !sp_idx) || !(sampling->temperature > 0.f) || sampling->top_k < 0)) return SSD_ERR_BAD_ARG;
     const ssd_config &c = ctx->cfg;
     int32_t depth[SSD_MAX_NODES];
     int max_depth = 0;
@@ -806,6 +809,7 @@ int ssd_accept_tree(ssd_ctx *ctx, const float *logits, const float *draft_probs,
     }
     int launched = 0;
     AcceptScratch sc = ctx->acc;
+    sc.sp_idx = sp_idx; sc.sp_val = sp_val; sc.sp_entries = sp_entries;
     sc.result = ctx->h_result; // the walk writes its few words straight into the pinned host buffer: no copy to enqueue and wait for
     sc.dev_status = ctx->d_status;
     // greedy on the very logits the last forward of this context wrote: the LM head's per-tile row statistics stand in for them
@@ -828,6 +832,13 @@ int ssd_accept_tree(ssd_ctx *ctx, const float *logits, const float *draft_probs,
     if (ctx->h_result[3] != 0) return SSD_ERR_TIMEOUT;
     return ctx->h_result[2];
 }
+} // namespace
+
+int ssd_accept_tree(ssd_ctx *ctx, const float *logits, const float *draft_probs, const int32_t *tokens, const int32_t *parent_idx,
+                    int32_t n_nodes, const ssd_sampling *sampling, ssd_rng *rng_state, int32_t *path_out, int32_t *n_path_out,
+                    int32_t *next_token_out) {
+    return accept_impl(ctx, logits, draft_probs, nullptr, nullptr, 0, tokens, parent_idx, n_nodes, sampling, rng_state, path_out, n_path_out, next_token_out);
+}
 
 int ssd_accept_tree_sparse(ssd_ctx *ctx, const float *logits, const int32_t *row_idx, const float *row_val, int32_t entries,
                            const int32_t *tokens, const int32_t *parent_idx, int32_t n_nodes, const ssd_sampling *sampling, ssd_rng *rng_state,
@@ -835,6 +846,7 @@ int ssd_accept_tree_sparse(ssd_ctx *ctx, const float *logits, const int32_t *row
     if (!ctx || !row_idx || !row_val || entries < 1 || entries > SSD_ACC_SUPPORT || n_nodes < 1 || n_nodes > SSD_MAX_NODES) return SSD_ERR_BAD_ARG;
     DeviceGuard g(ctx->device);
     if (!g.ok) return SSD_ERR_CUDA;
+    if (!sampling) return SSD_ERR_BAD_ARG;
     const size_t need_e = (size_t)n_nodes * entries, need_r = (size_t)n_nodes * ctx->cfg.vocab;
     if (ctx->sparse_entries_cap < need_e) {
         CU(cudaStreamSynchronize(ctx->stream));
@@ -844,6 +856,17 @@ int ssd_accept_tree_sparse(ssd_ctx *ctx, const float *logits, const int32_t *row
         CU(cudaMalloc((void **)&ctx->d_sparse_val, need_e * sizeof(float)));
         ctx->sparse_entries_cap = need_e;
     }
+    // (the lists are pageable host memory: the copies have read them by the time the calls return)
+    CU(cudaMemcpyAsync(ctx->d_sparse_idx, row_idx, need_e * sizeof(int32_t), cudaMemcpyHostToDevice, ctx->stream));
+    CU(cudaMemcpyAsync(ctx->d_sparse_val, row_val, need_e * sizeof(float), cudaMemcpyHostToDevice, ctx->stream));
+    // The decision kernels read the lists directly (a refusal then costs O(entries), not two passes over the vocabulary) whenever
+    // every node has a scratch row for its law - the normal case; a greedy walk reads no rows at all.
+    bool lists = sampling->mode == SSD_GREEDY;
+    if (sampling->mode == SSD_SAMPLING && n_nodes > 1) lists = ensure_law_rows(ctx, n_nodes) == SSD_OK && ctx->acc.rows_cap >= n_nodes;
+    if (lists || n_nodes == 1)
+        return accept_impl(ctx, logits, nullptr, ctx->d_sparse_idx, ctx->d_sparse_val, entries, tokens, parent_idx, n_nodes, sampling, rng_state, path_out,
+                           n_path_out, next_token_out);
+    // otherwise: expand to dense rows and take the one-CTA walk
     if (ctx->sparse_rows_cap < need_r) {
         CU(cudaStreamSynchronize(ctx->stream));
         cudaFree(ctx->d_sparse_rows);
@@ -851,11 +874,8 @@ int ssd_accept_tree_sparse(ssd_ctx *ctx, const float *logits, const int32_t *row
         CU(cudaMalloc((void **)&ctx->d_sparse_rows, need_r * sizeof(float)));
         ctx->sparse_rows_cap = need_r;
     }
-    CU(cudaMemcpyAsync(ctx->d_sparse_idx, row_idx, need_e * sizeof(int32_t), cudaMemcpyHostToDevice, ctx->stream));
-    CU(cudaMemcpyAsync(ctx->d_sparse_val, row_val, need_e * sizeof(float), cudaMemcpyHostToDevice, ctx->stream));
     CU(launch_expand_sparse_rows(ctx->d_sparse_idx, ctx->d_sparse_val, n_nodes, entries, ctx->cfg.vocab, ctx->d_sparse_rows, ctx->stream));
     ctx->launches += 1;
-    // (the lists are pageable host memory: the copies above have read them by the time the calls return)
     return ssd_accept_tree(ctx, logits, ctx->d_sparse_rows, tokens, parent_idx, n_nodes, sampling, rng_state, path_out, n_path_out, next_token_out);
 }
 

@@ -165,6 +165,10 @@ struct AcceptScratch {
     int32_t *row_bad;   // [max_nodes * parts] 1 if the part holds a non-finite value (sampling: [max_nodes], per row)
     int32_t *result;    // [max_nodes + 4]: n_path, next_token, status, device error word, path[...]
     const int32_t *dev_status; // the forward's device error word (copied into result[3] by the walk) or null
+    // sampling with the per-node scratch: proposal rows as index / value lists [n][sp_entries] (device) instead of dense rows; null = dense
+    const int32_t *sp_idx;
+    const float *sp_val;
+    int sp_entries;
     // greedy: per (row, part) statistics already written by the LM head (parts = head_parts > 0): the arg-max pass is skipped
     int head_parts;
     const float *head_val;
