@@ -194,7 +194,10 @@ __device__ float kth_largest(const float *__restrict__ z, int V, int k, BlockScr
 
 // Target law of one node, r[v] = softmax(z / T) over the kept entries (all, or the top_k largest logits, ties kept),
 // in fp64 by the whole CTA; returns 1 if the row holds a non-finite value (r is then unspecified).
-__device__ int row_law(const float *__restrict__ z, int V, double temperature, int top_k, double *__restrict__ r, BlockScratch &s) {
+// With `total` given the row is left UNNORMALISED (r[v] = exp(z[v] / T - max), *total = their sum, the same value in every thread):
+// the acceptance rule works on r and its total (see node_decide), which spares V fp64 divisions here and V more per refusal.
+__device__ int row_law(const float *__restrict__ z, int V, double temperature, int top_k, double *__restrict__ r, BlockScratch &s,
+                       double *total = nullptr) {
     const int tid = threadIdx.x;
     int bad = 0;
     for (int v = tid; v < V; v += ACC_THREADS) bad |= !isfinite(z[v]);
@@ -214,7 +217,9 @@ __device__ int row_law(const float *__restrict__ z, int V, double temperature, i
         part += p;
     }
     const double den = block_sum(part, s);
-    for (int v = tid; v < V; v += ACC_THREADS) r[v] /= den;
+    if (total) *total = den;
+    else
+        for (int v = tid; v < V; v += ACC_THREADS) r[v] /= den;
     __syncthreads();
     return 0;
 }
@@ -252,12 +257,13 @@ __device__ void list_support(const double *__restrict__ r, int V, int32_t *__res
 }
 
 __global__ void __launch_bounds__(ACC_THREADS) row_law_kernel(const float *__restrict__ logits, int V, double temperature, int top_k,
-                                                              double *__restrict__ rows, int32_t *__restrict__ row_bad,
+                                                              double *__restrict__ rows, double *__restrict__ row_total, int32_t *__restrict__ row_bad,
                                                               int32_t *__restrict__ sup_idx, int32_t *__restrict__ sup_cnt) {
     __shared__ BlockScratch s;
     const int row = blockIdx.x;
-    const int bad = row_law(logits + (size_t)row * V, V, temperature, top_k, rows + (size_t)row * V, s);
-    if (threadIdx.x == 0) row_bad[row] = bad;
+    double total = 1.0;
+    const int bad = row_law(logits + (size_t)row * V, V, temperature, top_k, rows + (size_t)row * V, s, &total);
+    if (threadIdx.x == 0) { row_bad[row] = bad; row_total[row] = total; }
     if (sup_cnt) {
         if (!bad && top_k > 0 && top_k < V) list_support(rows + (size_t)row * V, V, sup_idx + (size_t)row * SSD_ACC_SUPPORT, sup_cnt + row, s);
         else if (threadIdx.x == 0) sup_cnt[row] = -1;
@@ -313,10 +319,11 @@ __device__ void draw_from(const double *__restrict__ r, int V, double u, int32_t
 // the walk reached cur - so all nodes can be decided side by side.
 //
 // Proposal rows come dense (draft[c, :]) or as short lists (sp.idx / sp.val, [n][sp.entries], distinct indices, < 0 = unused).
-// With lists and a dense law a refusal touches the listed entries only: the residual max(0, r - q) differs from r there and
-// nowhere else, so r is kept UNNORMALISED with its total `norm` beside it (r_true = r / norm: the test u q[x] < r_true[x] becomes
-// u q[x] norm < r[x], the subtraction r - q norm, the new total norm minus what the listed entries lost) - O(entries) per refusal
-// instead of two passes over the vocabulary.  The extra token's inverse CDF sums r itself, so it needs no total.
+// r is UNNORMALISED throughout, its total `norm` beside it (r_true = r / norm): the test u q[x] < r_true[x] becomes
+// u q[x] norm < r[x], the residual max(0, r - q norm) with its own sum as the new total - no division anywhere.  With lists and a
+// dense law a refusal touches the listed entries only (the residual differs from r there and nowhere else; the new total is
+// norm minus what they lost): O(entries) per refusal instead of two passes over the vocabulary.  The extra token's inverse CDF
+// sums r itself, so it needs no total.
 struct SparseRows { const int32_t *idx; const float *val; int entries; };
 __device__ __forceinline__ float q_at(const float *__restrict__ draft, const SparseRows &sp, int c, int V, int v) {
     if (!sp.idx) return draft[(size_t)c * V + v];
@@ -326,9 +333,8 @@ __device__ __forceinline__ float q_at(const float *__restrict__ draft, const Spa
 }
 __device__ int node_decide(double *__restrict__ r, int cnt, const int32_t *__restrict__ sup, const float *__restrict__ draft, const SparseRows sp,
                            const NodeList &tokens, const NodeList &parent, int n, int V, uint64_t seed, uint64_t step, int cur,
-                           int32_t *__restrict__ token_out, BlockScratch &s) {
+                           int32_t *__restrict__ token_out, BlockScratch &s, double norm) { // norm: the total of r on entry
     const int tid = threadIdx.x;
-    double norm = 1.0; // total of r (lists with a dense law; every other case renormalises r in place and keeps 1)
     for (int c = cur + 1; c < n; ++c) {
         if (parent.v[c] != cur) continue;
         const float *q = draft ? draft + (size_t)c * V : nullptr;
@@ -339,9 +345,12 @@ __device__ int node_decide(double *__restrict__ r, int cnt, const int32_t *__res
         __syncthreads(); // all threads have read r[x] before anyone rewrites it
         if (cnt >= 0) { // one support entry per thread
             const int iv = tid < cnt ? sup[tid] : 0;
-            const double val = tid < cnt ? fmax(r[iv] - (double)q_at(draft, sp, c, V, iv), 0.0) : 0.0;
+            const double val = tid < cnt ? fmax(r[iv] - (double)q_at(draft, sp, c, V, iv) * norm, 0.0) : 0.0;
             const double Z = block_sum(val, s);
-            if (Z > 0.0 && tid < cnt) r[iv] = val / Z;
+            if (Z > 0.0) {
+                if (tid < cnt) r[iv] = val;
+                norm = Z;
+            }
         } else if (sp.idx) { // listed entries only
             double lost = 0.0;
             for (int e = tid; e < sp.entries; e += ACC_THREADS) {
@@ -358,10 +367,12 @@ __device__ int node_decide(double *__restrict__ r, int cnt, const int32_t *__res
             }
         } else {
             double zs = 0.0;
-            for (int v = tid; v < V; v += ACC_THREADS) zs += fmax(r[v] - (double)q[v], 0.0);
+            for (int v = tid; v < V; v += ACC_THREADS) zs += fmax(r[v] - (double)q[v] * norm, 0.0);
             const double Z = block_sum(zs, s);
-            if (Z > 0.0)
-                for (int v = tid; v < V; v += ACC_THREADS) r[v] = fmax(r[v] - (double)q[v], 0.0) / Z;
+            if (Z > 0.0) {
+                for (int v = tid; v < V; v += ACC_THREADS) r[v] = fmax(r[v] - (double)q[v] * norm, 0.0);
+                norm = Z;
+            }
         }
         __syncthreads();
     }
@@ -403,11 +414,12 @@ __global__ void __launch_bounds__(ACC_THREADS) sample_walk_kernel(const float *_
     if (tid == 0) { result[3] = dev_status ? *dev_status : 0; result[4] = 0; }
     for (;;) {
         // a visited row must be finite
-        if (row_law(logits + (size_t)cur * V, V, temperature, top_k, r, s)) {
+        double total = 1.0;
+        if (row_law(logits + (size_t)cur * V, V, temperature, top_k, r, s, &total)) {
             if (tid == 0) { result[0] = 1; result[1] = -1; result[2] = SSD_ERR_BAD_ARG; }
             return;
         }
-        const int c = node_decide(r, -1, nullptr, draft, SparseRows{nullptr, nullptr, 0}, tokens, parent, n, V, seed, step, cur, result + 1, s);
+        const int c = node_decide(r, -1, nullptr, draft, SparseRows{nullptr, nullptr, 0}, tokens, parent, n, V, seed, step, cur, result + 1, s, total);
         if (c < 0) {
             if (tid == 0) { result[0] = np; result[2] = SSD_OK; }
             return;
@@ -423,7 +435,7 @@ __global__ void __launch_bounds__(ACC_THREADS) sample_walk_kernel(const float *_
 // token), -2 if p's logits are unusable.
 __global__ void __launch_bounds__(ACC_THREADS) node_decide_kernel(const float *__restrict__ draft, SparseRows sp, NodeList tokens, NodeList parent, int n, int V,
                                                                   uint64_t seed, uint64_t step, double *__restrict__ rows,
-                                                                  const int32_t *__restrict__ row_bad, const int32_t *__restrict__ sup_idx,
+                                                                  const double *__restrict__ row_total, const int32_t *__restrict__ row_bad, const int32_t *__restrict__ sup_idx,
                                                                   const int32_t *__restrict__ sup_cnt, int32_t *__restrict__ next,
                                                                   int32_t *__restrict__ bonus) {
     __shared__ BlockScratch s;
@@ -434,7 +446,7 @@ __global__ void __launch_bounds__(ACC_THREADS) node_decide_kernel(const float *_
     }
     const int cnt = sup_cnt ? sup_cnt[p] : -1;
     const int c = node_decide(rows + (size_t)p * V, cnt, cnt >= 0 ? sup_idx + (size_t)p * SSD_ACC_SUPPORT : nullptr, draft, sp, tokens, parent, n, V,
-                              seed, step, p, bonus + p, s);
+                              seed, step, p, bonus + p, s, row_total[p]);
     if (threadIdx.x == 0) next[p] = c;
 }
 
@@ -473,9 +485,9 @@ cudaError_t launch_accept(const float *logits, const float *draft_probs, const N
         if (rows) {
             // every node is decided by a CTA of its own (its law, then its children in order), then a walk follows the decisions
             int32_t *next = sc.row_arg, *bonus = sc.row_arg + n; // (row_arg holds 4 ints per node on this path)
-            row_law_kernel<<<n, ACC_THREADS, 0, s>>>(logits, vocab, (double)temperature, top_k, rows, sc.row_bad, sc.sup_idx, sc.sup_cnt);
+            row_law_kernel<<<n, ACC_THREADS, 0, s>>>(logits, vocab, (double)temperature, top_k, rows, sc.row_total, sc.row_bad, sc.sup_idx, sc.sup_cnt);
             const SparseRows sp = {sc.sp_idx, sc.sp_val, sc.sp_entries}; // (lists instead of dense rows: draft_probs is then not read)
-            node_decide_kernel<<<n, ACC_THREADS, 0, s>>>(draft_probs, sp, tokens, parent, n, vocab, seed, step, rows, sc.row_bad, sc.sup_idx, sc.sup_cnt,
+            node_decide_kernel<<<n, ACC_THREADS, 0, s>>>(draft_probs, sp, tokens, parent, n, vocab, seed, step, rows, sc.row_total, sc.row_bad, sc.sup_idx, sc.sup_cnt,
                                                          next, bonus);
             chain_walk_kernel<<<1, 32, 0, s>>>(next, bonus, n, sc.result, sc.dev_status);
             *launches += 3;

@@ -400,8 +400,9 @@ int ensure_law_rows(ssd_ctx *ctx, int n) {
     const int rows = (n + 31) & ~31;
     const size_t law_bytes = (size_t)rows * ctx->cfg.vocab * sizeof(double), idx_bytes = (size_t)rows * SSD_ACC_SUPPORT * sizeof(int32_t);
     void *q = nullptr;
-    if (cudaMalloc(&q, law_bytes + idx_bytes + (size_t)rows * sizeof(int32_t)) == cudaSuccess) {
+    if (cudaMalloc(&q, law_bytes + idx_bytes + (size_t)rows * sizeof(int32_t) + (size_t)rows * sizeof(double) + 8) == cudaSuccess) {
         ctx->acc.rows = (double *)q; ctx->acc.rows_cap = rows;
+        ctx->acc.row_total = (double *)(((uintptr_t)q + law_bytes + idx_bytes + (size_t)rows * sizeof(int32_t) + 7) & ~(uintptr_t)7);
         ctx->acc.sup_idx = (int32_t *)((char *)q + law_bytes);
         ctx->acc.sup_cnt = (int32_t *)((char *)q + law_bytes + idx_bytes);
     } else {

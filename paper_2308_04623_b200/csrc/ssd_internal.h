@@ -156,6 +156,7 @@ struct AcceptScratch {
     double *rows;       // [rows_cap, vocab] target distribution of every node, computed by one CTA per row before the walk
                         // (null or too small: the walk computes the visited rows itself, one after the other)
     int rows_cap;
+    double *row_total;  // [rows_cap] the rows are unnormalised: their totals
     int32_t *sup_idx;   // [rows_cap, SSD_ACC_SUPPORT] with a top-k cut: the indices a row's law is positive at, ascending
     int32_t *sup_cnt;   // [rows_cap] how many (-1: more than SSD_ACC_SUPPORT, the walk then scans the whole vocabulary)
     double *r;          // [vocab] residual distribution
