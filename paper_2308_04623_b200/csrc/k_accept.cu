@@ -516,14 +516,15 @@ __global__ void __launch_bounds__(ACC_THREADS) propose_children_kernel(const flo
     __shared__ int32_t s_pick;
     const int j = blockIdx.x, node = nodes.v[j], tid = threadIdx.x;
     double *r = scratch + (size_t)j * V;
-    const int bad = row_law(logits + (size_t)node * V, V, temperature, top_k, r, s);
+    double total = 1.0; // (r stays unnormalised: the picks and draws do not need it otherwise, the row written out is divided on its way)
+    const int bad = row_law(logits + (size_t)node * V, V, temperature, top_k, r, s, &total);
     if (tid == 0) bad_out[j] = bad;
     if (bad) {
         for (int t = tid; t < picks; t += ACC_THREADS) tokens_out[j * picks + t] = -1;
         return;
     }
     if (rows_out)
-        for (int v = tid; v < V; v += ACC_THREADS) rows_out[(size_t)j * V + v] = (float)r[v];
+        for (int v = tid; v < V; v += ACC_THREADS) rows_out[(size_t)j * V + v] = (float)(r[v] / total);
     for (int t = 0; t < picks; ++t) {
         if (mode == SSD_GREEDY) { // the most probable token not yet picked; ties towards the lower id
             double best = -1.0;
