@@ -199,17 +199,18 @@ __device__ float kth_largest(const float *__restrict__ z, int V, int k, BlockScr
 __device__ int row_law(const float *__restrict__ z, int V, double temperature, int top_k, double *__restrict__ r, BlockScratch &s,
                        double *total = nullptr) {
     const int tid = threadIdx.x;
+    // one pass for the finiteness check and the maximum (the largest entry survives any top-k cut, and dividing by a positive
+    // temperature keeps the order: the maximum of the kept z / T is z_max / T)
     int bad = 0;
-    for (int v = tid; v < V; v += ACC_THREADS) bad |= !isfinite(z[v]);
+    float zmax = -INFINITY;
+    for (int v = tid; v < V; v += ACC_THREADS) { const float zv = z[v]; bad |= !isfinite(zv); zmax = fmaxf(zmax, zv); }
     if (block_max_int(bad, s)) return 1;
     float thr = -INFINITY;
     if (top_k > 0 && top_k < V) thr = kth_largest(z, V, top_k, s);
     // (x / 1.0 is x exactly: at temperature 1 the fp64 division, a large part of this function's time, is skipped)
     const bool unit_t = temperature == 1.0;
-    double mx = -INFINITY;
-    for (int v = tid; v < V; v += ACC_THREADS)
-        if (z[v] >= thr) mx = fmax(mx, unit_t ? (double)z[v] : (double)z[v] / temperature);
-    mx = block_max(mx, s);
+    const double zm = block_max((double)zmax, s);
+    const double mx = unit_t ? zm : zm / temperature;
     double part = 0.0;
     for (int v = tid; v < V; v += ACC_THREADS) {
         const double p = (z[v] >= thr) ? exp((unit_t ? (double)z[v] : (double)z[v] / temperature) - mx) : 0.0;
