@@ -196,8 +196,11 @@ __device__ float kth_largest(const float *__restrict__ z, int V, int k, BlockScr
 // in fp64 by the whole CTA; returns 1 if the row holds a non-finite value (r is then unspecified).
 // With `total` given the row is left UNNORMALISED (r[v] = exp(z[v] / T - max), *total = their sum, the same value in every thread):
 // the acceptance rule works on r and its total (see node_decide), which spares V fp64 divisions here and V more per refusal.
+// The exponentials are what the law costs (fp64, ~60 multiply-adds each, at an SM's fp64 rate some 20 us for a GPT-2
+// vocabulary), so a row can be cut into `parts` slices for as many CTAs: each looks at the whole row for the checks, the
+// maximum and the cut, exponentiates its own slice only and returns that slice's sum (unnormalised rows only).
 __device__ int row_law(const float *__restrict__ z, int V, double temperature, int top_k, double *__restrict__ r, BlockScratch &s,
-                       double *total = nullptr) {
+                       double *total = nullptr, int part = 0, int parts = 1) {
     const int tid = threadIdx.x;
     // one pass for the finiteness check and the maximum (the largest entry survives any top-k cut, and dividing by a positive
     // temperature keeps the order: the maximum of the kept z / T is z_max / T)
@@ -211,13 +214,14 @@ __device__ int row_law(const float *__restrict__ z, int V, double temperature, i
     const bool unit_t = temperature == 1.0;
     const double zm = block_max((double)zmax, s);
     const double mx = unit_t ? zm : zm / temperature;
-    double part = 0.0;
-    for (int v = tid; v < V; v += ACC_THREADS) {
+    double acc = 0.0;
+    const int v0 = (int)(((long long)V * part) / parts), v1 = (int)(((long long)V * (part + 1)) / parts);
+    for (int v = v0 + tid; v < v1; v += ACC_THREADS) {
         const double p = (z[v] >= thr) ? exp((unit_t ? (double)z[v] : (double)z[v] / temperature) - mx) : 0.0;
         r[v] = p;
-        part += p;
+        acc += p;
     }
-    const double den = block_sum(part, s);
+    const double den = block_sum(acc, s);
     if (total) *total = den;
     else
         for (int v = tid; v < V; v += ACC_THREADS) r[v] /= den;
@@ -257,18 +261,28 @@ __device__ void list_support(const double *__restrict__ r, int V, int32_t *__res
     __syncthreads();
 }
 
-__global__ void __launch_bounds__(ACC_THREADS) row_law_kernel(const float *__restrict__ logits, int V, double temperature, int top_k,
-                                                              double *__restrict__ rows, double *__restrict__ row_total, int32_t *__restrict__ row_bad,
-                                                              int32_t *__restrict__ sup_idx, int32_t *__restrict__ sup_cnt) {
+constexpr int ACC_MAX_PARTS = 8; // slices a row's law is computed in (one CTA each)
+__global__ void __launch_bounds__(ACC_THREADS) row_law_kernel(const float *__restrict__ logits, NodeList nodes, int use_list, int V, double temperature,
+                                                              int top_k, double *__restrict__ rows, double *__restrict__ row_total,
+                                                              int32_t *__restrict__ row_bad) {
     __shared__ BlockScratch s;
-    const int row = blockIdx.x;
+    const int row = blockIdx.x, node = use_list ? nodes.v[row] : row;
     double total = 1.0;
-    const int bad = row_law(logits + (size_t)row * V, V, temperature, top_k, rows + (size_t)row * V, s, &total);
-    if (threadIdx.x == 0) { row_bad[row] = bad; row_total[row] = total; }
-    if (sup_cnt) {
-        if (!bad && top_k > 0 && top_k < V) list_support(rows + (size_t)row * V, V, sup_idx + (size_t)row * SSD_ACC_SUPPORT, sup_cnt + row, s);
-        else if (threadIdx.x == 0) sup_cnt[row] = -1;
+    const int bad = row_law(logits + (size_t)node * V, V, temperature, top_k, rows + (size_t)row * V, s, &total, blockIdx.y, gridDim.y);
+    if (threadIdx.x == 0) {
+        row_total[row * ACC_MAX_PARTS + blockIdx.y] = total;
+        if (blockIdx.y == 0) row_bad[row] = bad; // (every slice sees the whole row: the same verdict)
     }
+}
+// The row's total from its slices' sums, in slice order (the same value in every thread and in every run).
+__device__ __forceinline__ double row_total_of(const double *__restrict__ row_total, int row, int parts) {
+    double t = 0.0;
+    for (int p = 0; p < parts; ++p) t += row_total[row * ACC_MAX_PARTS + p];
+    return t;
+}
+inline int law_parts(int rows) { // as many slices as keep all CTAs of the launch on the GPU at once
+    int p = 148 / (rows > 0 ? rows : 1);
+    return p < 1 ? 1 : (p > ACC_MAX_PARTS ? ACC_MAX_PARTS : p);
 }
 
 // Inverse-CDF draw from r (fp64, not necessarily normalised) by the whole CTA: ONE thread writes to *token_out the smallest v
@@ -436,8 +450,9 @@ __global__ void __launch_bounds__(ACC_THREADS) sample_walk_kernel(const float *_
 // token), -2 if p's logits are unusable.
 __global__ void __launch_bounds__(ACC_THREADS) node_decide_kernel(const float *__restrict__ draft, SparseRows sp, NodeList tokens, NodeList parent, int n, int V,
                                                                   uint64_t seed, uint64_t step, double *__restrict__ rows,
-                                                                  const double *__restrict__ row_total, const int32_t *__restrict__ row_bad, const int32_t *__restrict__ sup_idx,
-                                                                  const int32_t *__restrict__ sup_cnt, int32_t *__restrict__ next,
+                                                                  const double *__restrict__ row_total, int parts, int cut,
+                                                                  const int32_t *__restrict__ row_bad, int32_t *__restrict__ sup_idx,
+                                                                  int32_t *__restrict__ sup_cnt, int32_t *__restrict__ next,
                                                                   int32_t *__restrict__ bonus) {
     __shared__ BlockScratch s;
     const int p = blockIdx.x;
@@ -445,9 +460,16 @@ __global__ void __launch_bounds__(ACC_THREADS) node_decide_kernel(const float *_
         if (threadIdx.x == 0) next[p] = -2;
         return;
     }
+    // with a top-k cut the law is positive at few indices: list them (ascending), so that the residual updates and the
+    // inverse-CDF scan touch those entries only
+    if (sup_cnt) {
+        if (cut) list_support(rows + (size_t)p * V, V, sup_idx + (size_t)p * SSD_ACC_SUPPORT, sup_cnt + p, s);
+        else if (threadIdx.x == 0) sup_cnt[p] = -1;
+        __syncthreads();
+    }
     const int cnt = sup_cnt ? sup_cnt[p] : -1;
     const int c = node_decide(rows + (size_t)p * V, cnt, cnt >= 0 ? sup_idx + (size_t)p * SSD_ACC_SUPPORT : nullptr, draft, sp, tokens, parent, n, V,
-                              seed, step, p, bonus + p, s, row_total[p]);
+                              seed, step, p, bonus + p, s, row_total_of(row_total, p, parts));
     if (threadIdx.x == 0) next[p] = c;
 }
 
@@ -486,10 +508,11 @@ cudaError_t launch_accept(const float *logits, const float *draft_probs, const N
         if (rows) {
             // every node is decided by a CTA of its own (its law, then its children in order), then a walk follows the decisions
             int32_t *next = sc.row_arg, *bonus = sc.row_arg + n; // (row_arg holds 4 ints per node on this path)
-            row_law_kernel<<<n, ACC_THREADS, 0, s>>>(logits, vocab, (double)temperature, top_k, rows, sc.row_total, sc.row_bad, sc.sup_idx, sc.sup_cnt);
+            const int parts = law_parts(n);
+            row_law_kernel<<<dim3(n, parts), ACC_THREADS, 0, s>>>(logits, tokens, 0, vocab, (double)temperature, top_k, rows, sc.row_total, sc.row_bad);
             const SparseRows sp = {sc.sp_idx, sc.sp_val, sc.sp_entries}; // (lists instead of dense rows: draft_probs is then not read)
-            node_decide_kernel<<<n, ACC_THREADS, 0, s>>>(draft_probs, sp, tokens, parent, n, vocab, seed, step, rows, sc.row_total, sc.row_bad, sc.sup_idx, sc.sup_cnt,
-                                                         next, bonus);
+            node_decide_kernel<<<n, ACC_THREADS, 0, s>>>(draft_probs, sp, tokens, parent, n, vocab, seed, step, rows, sc.row_total, parts, (top_k > 0 && top_k < vocab) ? 1 : 0,
+                                                         sc.row_bad, sc.sup_idx, sc.sup_cnt, next, bonus);
             chain_walk_kernel<<<1, 32, 0, s>>>(next, bonus, n, sc.result, sc.dev_status);
             *launches += 3;
         } else {
@@ -511,14 +534,17 @@ cudaError_t launch_accept(const float *logits, const float *draft_probs, const N
 // ---------------------------------------------------------------------------------------------
 __global__ void __launch_bounds__(ACC_THREADS) propose_children_kernel(const float *__restrict__ logits, NodeList nodes, int V, double temperature,
                                                                        int top_k, int mode, int picks, uint64_t seed, uint64_t step,
-                                                                       double *__restrict__ scratch, float *__restrict__ rows_out,
+                                                                       double *__restrict__ scratch, const double *__restrict__ row_total, int parts,
+                                                                       const int32_t *__restrict__ row_bad, float *__restrict__ rows_out,
                                                                        int32_t *__restrict__ tokens_out, int32_t *__restrict__ bad_out) {
     __shared__ BlockScratch s;
     __shared__ int32_t s_pick;
     const int j = blockIdx.x, node = nodes.v[j], tid = threadIdx.x;
     double *r = scratch + (size_t)j * V;
-    double total = 1.0; // (r stays unnormalised: the picks and draws do not need it otherwise, the row written out is divided on its way)
-    const int bad = row_law(logits + (size_t)node * V, V, temperature, top_k, r, s, &total);
+    // (row_law_kernel has left the law of listed node j in scratch row j, unnormalised: the picks and draws do not need it
+    //  otherwise, the row written out is divided on its way)
+    const double total = row_total_of(row_total, j, parts);
+    const int bad = row_bad[j];
     if (tid == 0) bad_out[j] = bad;
     if (bad) {
         for (int t = tid; t < picks; t += ACC_THREADS) tokens_out[j * picks + t] = -1;
@@ -546,10 +572,12 @@ __global__ void __launch_bounds__(ACC_THREADS) propose_children_kernel(const flo
 }
 
 cudaError_t launch_propose_children(const float *logits, const NodeList &nodes, int m, int vocab, int mode, float temperature, int top_k, int picks,
-                                    uint64_t seed, uint64_t step, double *scratch, float *rows_out, int32_t *tokens_out, int32_t *bad_out,
-                                    cudaStream_t s) {
-    propose_children_kernel<<<m, ACC_THREADS, 0, s>>>(logits, nodes, vocab, (double)temperature, top_k, mode, picks, seed, step, scratch, rows_out,
-                                                      tokens_out, bad_out);
+                                    uint64_t seed, uint64_t step, double *scratch, double *row_total, int32_t *row_bad, float *rows_out,
+                                    int32_t *tokens_out, int32_t *bad_out, cudaStream_t s) {
+    const int parts = law_parts(m);
+    row_law_kernel<<<dim3(m, parts), ACC_THREADS, 0, s>>>(logits, nodes, 1, vocab, (double)temperature, top_k, scratch, row_total, row_bad);
+    propose_children_kernel<<<m, ACC_THREADS, 0, s>>>(logits, nodes, vocab, (double)temperature, top_k, mode, picks, seed, step, scratch, row_total, parts,
+                                                      row_bad, rows_out, tokens_out, bad_out);
     return cudaGetLastError();
 }
 

@@ -400,7 +400,7 @@ int ensure_law_rows(ssd_ctx *ctx, int n) {
     const int rows = (n + 31) & ~31;
     const size_t law_bytes = (size_t)rows * ctx->cfg.vocab * sizeof(double), idx_bytes = (size_t)rows * SSD_ACC_SUPPORT * sizeof(int32_t);
     void *q = nullptr;
-    if (cudaMalloc(&q, law_bytes + idx_bytes + (size_t)rows * sizeof(int32_t) + (size_t)rows * sizeof(double) + 8) == cudaSuccess) {
+    if (cudaMalloc(&q, law_bytes + idx_bytes + (size_t)rows * sizeof(int32_t) + (size_t)rows * 8 * sizeof(double) + 8) == cudaSuccess) {
         ctx->acc.rows = (double *)q; ctx->acc.rows_cap = rows;
         ctx->acc.row_total = (double *)(((uintptr_t)q + law_bytes + idx_bytes + (size_t)rows * sizeof(int32_t) + 7) & ~(uintptr_t)7);
         ctx->acc.sup_idx = (int32_t *)((char *)q + law_bytes);
@@ -896,8 +896,8 @@ int ssd_propose_children(ssd_ctx *ctx, const float *logits, const int32_t *nodes
     memcpy(nl.v, nodes, sizeof(int32_t) * m);
     int32_t *picks_host = ctx->h_propose, *bad_host = ctx->h_propose + SSD_MAX_NODES * 8; // the kernel writes into pinned host memory
     CU(launch_propose_children(logits, nl, m, ctx->cfg.vocab, sampling->mode, sampling->temperature, sampling->top_k, picks, rng_state->seed,
-                               rng_state->step, ctx->acc.rows, rows_out, picks_host, bad_host, ctx->stream));
-    ctx->launches += 1;
+                               rng_state->step, ctx->acc.rows, ctx->acc.row_total, ctx->acc.row_bad, rows_out, picks_host, bad_host, ctx->stream));
+    ctx->launches += 2;
     CU(cudaStreamSynchronize(ctx->stream));
     rng_state->step += 1;
     for (int j = 0; j < m; ++j)

@@ -156,7 +156,7 @@ struct AcceptScratch {
     double *rows;       // [rows_cap, vocab] target distribution of every node, computed by one CTA per row before the walk
                         // (null or too small: the walk computes the visited rows itself, one after the other)
     int rows_cap;
-    double *row_total;  // [rows_cap] the rows are unnormalised: their totals
+    double *row_total;  // [rows_cap][8] the rows are unnormalised: the sums of the (up to eight) slices they were computed in
     int32_t *sup_idx;   // [rows_cap, SSD_ACC_SUPPORT] with a top-k cut: the indices a row's law is positive at, ascending
     int32_t *sup_cnt;   // [rows_cap] how many (-1: more than SSD_ACC_SUPPORT, the walk then scans the whole vocabulary)
     double *r;          // [vocab] residual distribution
@@ -176,8 +176,8 @@ struct AcceptScratch {
     const int32_t *head_arg, *head_bad;
 };
 cudaError_t launch_propose_children(const float *logits, const NodeList &nodes, int m, int vocab, int mode, float temperature, int top_k, int picks,
-                                    uint64_t seed, uint64_t step, double *scratch, float *rows_out, int32_t *tokens_out, int32_t *bad_out,
-                                    cudaStream_t s);
+                                    uint64_t seed, uint64_t step, double *scratch, double *row_total, int32_t *row_bad, float *rows_out,
+                                    int32_t *tokens_out, int32_t *bad_out, cudaStream_t s);
 cudaError_t launch_expand_sparse_rows(const int32_t *idx, const float *val, int n, int entries, int vocab, float *rows, cudaStream_t s);
 cudaError_t launch_expired_wait(int32_t *status, long long limit_cycles, cudaStream_t s);
 cudaError_t launch_accept(const float *logits, const float *draft_probs, const NodeList &tokens, const NodeList &parent, int n,
