@@ -346,9 +346,10 @@ __device__ __forceinline__ float q_at(const float *__restrict__ draft, const Spa
         if (sp.idx[(size_t)c * sp.entries + e] == v) return sp.val[(size_t)c * sp.entries + e];
     return 0.f;
 }
-__device__ int node_decide(double *__restrict__ r, int cnt, const int32_t *__restrict__ sup, const float *__restrict__ draft, const SparseRows sp,
+__device__ int node_decide(double *r, int cnt, const int32_t *__restrict__ sup, const float *__restrict__ draft, const SparseRows sp,
                            const NodeList &tokens, const NodeList &parent, int n, int V, uint64_t seed, uint64_t step, int cur,
-                           int32_t *__restrict__ token_out, BlockScratch &s, double norm) { // norm: the total of r on entry
+                           int32_t *__restrict__ token_out, BlockScratch &s, double norm, double *r_alt = nullptr) {
+    // (norm: the total of r on entry; r_alt: a second row of V values, or null)
     const int tid = threadIdx.x;
     for (int c = cur + 1; c < n; ++c) {
         if (parent.v[c] != cur) continue;
@@ -382,11 +383,17 @@ __device__ int node_decide(double *__restrict__ r, int cnt, const int32_t *__res
             }
         } else {
             double zs = 0.0;
-            for (int v = tid; v < V; v += ACC_THREADS) zs += fmax(r[v] - (double)q[v] * norm, 0.0);
-            const double Z = block_sum(zs, s);
-            if (Z > 0.0) {
-                for (int v = tid; v < V; v += ACC_THREADS) r[v] = fmax(r[v] - (double)q[v] * norm, 0.0);
-                norm = Z;
+            if (r_alt) { // one pass: the residual goes to the other row while it is summed, and becomes r only if something is left
+                for (int v = tid; v < V; v += ACC_THREADS) { const double nv = fmax(r[v] - (double)q[v] * norm, 0.0); r_alt[v] = nv; zs += nv; }
+                const double Z = block_sum(zs, s);
+                if (Z > 0.0) { double *t = r; r = r_alt; r_alt = t; norm = Z; }
+            } else {
+                for (int v = tid; v < V; v += ACC_THREADS) zs += fmax(r[v] - (double)q[v] * norm, 0.0);
+                const double Z = block_sum(zs, s);
+                if (Z > 0.0) {
+                    for (int v = tid; v < V; v += ACC_THREADS) r[v] = fmax(r[v] - (double)q[v] * norm, 0.0);
+                    norm = Z;
+                }
             }
         }
         __syncthreads();
@@ -449,7 +456,7 @@ __global__ void __launch_bounds__(ACC_THREADS) sample_walk_kernel(const float *_
 // One CTA per node, after row_law_kernel: next[p] = the child accepted at p, -1 if none (bonus[p] then holds the extra
 // token), -2 if p's logits are unusable.
 __global__ void __launch_bounds__(ACC_THREADS) node_decide_kernel(const float *__restrict__ draft, SparseRows sp, NodeList tokens, NodeList parent, int n, int V,
-                                                                  uint64_t seed, uint64_t step, double *__restrict__ rows,
+                                                                  uint64_t seed, uint64_t step, double *__restrict__ rows, double *__restrict__ rows_alt,
                                                                   const double *__restrict__ row_total, int parts, int cut,
                                                                   const int32_t *__restrict__ row_bad, int32_t *__restrict__ sup_idx,
                                                                   int32_t *__restrict__ sup_cnt, int32_t *__restrict__ next,
@@ -469,7 +476,7 @@ __global__ void __launch_bounds__(ACC_THREADS) node_decide_kernel(const float *_
     }
     const int cnt = sup_cnt ? sup_cnt[p] : -1;
     const int c = node_decide(rows + (size_t)p * V, cnt, cnt >= 0 ? sup_idx + (size_t)p * SSD_ACC_SUPPORT : nullptr, draft, sp, tokens, parent, n, V,
-                              seed, step, p, bonus + p, s, row_total_of(row_total, p, parts));
+                              seed, step, p, bonus + p, s, row_total_of(row_total, p, parts), rows_alt ? rows_alt + (size_t)p * V : nullptr);
     if (threadIdx.x == 0) next[p] = c;
 }
 
@@ -511,7 +518,7 @@ cudaError_t launch_accept(const float *logits, const float *draft_probs, const N
             const int parts = law_parts(n);
             row_law_kernel<<<dim3(n, parts), ACC_THREADS, 0, s>>>(logits, tokens, 0, vocab, (double)temperature, top_k, rows, sc.row_total, sc.row_bad);
             const SparseRows sp = {sc.sp_idx, sc.sp_val, sc.sp_entries}; // (lists instead of dense rows: draft_probs is then not read)
-            node_decide_kernel<<<n, ACC_THREADS, 0, s>>>(draft_probs, sp, tokens, parent, n, vocab, seed, step, rows, sc.row_total, parts, (top_k > 0 && top_k < vocab) ? 1 : 0,
+            node_decide_kernel<<<n, ACC_THREADS, 0, s>>>(draft_probs, sp, tokens, parent, n, vocab, seed, step, rows, sc.rows_alt, sc.row_total, parts, (top_k > 0 && top_k < vocab) ? 1 : 0,
                                                          sc.row_bad, sc.sup_idx, sc.sup_cnt, next, bonus);
             chain_walk_kernel<<<1, 32, 0, s>>>(next, bonus, n, sc.result, sc.dev_status);
             *launches += 3;
@@ -662,7 +669,7 @@ cudaError_t noalloc_setup(int device, AcceptScratch *out) {
         slot.sc.result = (int32_t *)res;
         slot.sc.dev_status = nullptr;
         slot.sc.head_parts = 0;
-        slot.sc.sp_idx = nullptr; slot.sc.sp_val = nullptr; slot.sc.sp_entries = 0;
+        slot.sc.sp_idx = nullptr; slot.sc.sp_val = nullptr; slot.sc.sp_entries = 0; slot.sc.rows_alt = nullptr;
         slot.ready = true;
     }
     *out = slot.sc;

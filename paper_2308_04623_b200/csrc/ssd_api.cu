@@ -397,6 +397,7 @@ int ensure_law_rows(ssd_ctx *ctx, int n) {
     if (ctx->acc.rows_cap >= n) return SSD_OK;
     CU(cudaStreamSynchronize(ctx->stream));
     if (ctx->acc.rows) { cudaFree(ctx->acc.rows); ctx->acc.rows = nullptr; ctx->acc.rows_cap = 0; ctx->acc.sup_idx = ctx->acc.sup_cnt = nullptr; }
+    if (ctx->acc.rows_alt) { cudaFree(ctx->acc.rows_alt); ctx->acc.rows_alt = nullptr; }
     const int rows = (n + 31) & ~31;
     const size_t law_bytes = (size_t)rows * ctx->cfg.vocab * sizeof(double), idx_bytes = (size_t)rows * SSD_ACC_SUPPORT * sizeof(int32_t);
     void *q = nullptr;
@@ -405,6 +406,9 @@ int ensure_law_rows(ssd_ctx *ctx, int n) {
         ctx->acc.row_total = (double *)(((uintptr_t)q + law_bytes + idx_bytes + (size_t)rows * sizeof(int32_t) + 7) & ~(uintptr_t)7);
         ctx->acc.sup_idx = (int32_t *)((char *)q + law_bytes);
         ctx->acc.sup_cnt = (int32_t *)((char *)q + law_bytes + idx_bytes);
+        void *alt = nullptr; // (optional: without it a refusal takes two passes)
+        if (cudaMalloc(&alt, law_bytes) == cudaSuccess) ctx->acc.rows_alt = (double *)alt;
+        else (void)cudaGetLastError();
     } else {
         (void)cudaGetLastError();
     }
@@ -554,6 +558,7 @@ void ssd_destroy(ssd_ctx *ctx) {
     if (ctx->capture_stream) cudaStreamDestroy(ctx->capture_stream);
     for (void *p : ctx->owned) cudaFree(p);
     if (ctx->acc.rows) cudaFree(ctx->acc.rows);
+    if (ctx->acc.rows_alt) cudaFree(ctx->acc.rows_alt);
     if (ctx->h_result) cudaFreeHost(ctx->h_result);
     if (ctx->h_propose) cudaFreeHost(ctx->h_propose);
     cudaFree(ctx->d_sparse_idx); cudaFree(ctx->d_sparse_val); cudaFree(ctx->d_sparse_rows);

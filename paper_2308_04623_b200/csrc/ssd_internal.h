@@ -156,6 +156,7 @@ struct AcceptScratch {
     double *rows;       // [rows_cap, vocab] target distribution of every node, computed by one CTA per row before the walk
                         // (null or too small: the walk computes the visited rows itself, one after the other)
     int rows_cap;
+    double *rows_alt;   // [rows_cap, vocab] a second row per node (a refusal writes the residual there in one pass), or null
     double *row_total;  // [rows_cap][8] the rows are unnormalised: the sums of the (up to eight) slices they were computed in
     int32_t *sup_idx;   // [rows_cap, SSD_ACC_SUPPORT] with a top-k cut: the indices a row's law is positive at, ascending
     int32_t *sup_cnt;   // [rows_cap] how many (-1: more than SSD_ACC_SUPPORT, the walk then scans the whole vocabulary)
