@@ -46,6 +46,30 @@ def _run(name, P, trees, seed=0, chunk=256, **pair_args):
                 if (path, nxt) != (opath, onxt):
                     assert margin < 1e-9, (label, top_k, margin)
                     fragile += 1
+            # the same with proposal rows as four-entry lists (what a trigram stage hands over): the kernels read the lists, the
+            # oracle the dense rows they stand for; several steps, so that chains of refusals occur
+            n = len(tokens)
+            idx = np.argsort(-draft, axis=1)[:, :4].astype(np.int32)
+            idx[1:, 0] = tokens[1:]                      # (the proposed token is in its row's list, as a real proposal's is)
+            for c in range(1, n):                        # distinct indices per row
+                seen = set()
+                for e in range(4):
+                    while int(idx[c, e]) in seen:
+                        idx[c, e] = (idx[c, e] + 1) % p.V
+                    seen.add(int(idx[c, e]))
+            val = rng.dirichlet(np.ones(4), size=n).astype(np.float32)
+            dense = np.zeros((n, p.V), dtype=np.float32)
+            np.put_along_axis(dense, idx.astype(np.int64), val, axis=1)
+            for step in range(6):
+                for top_k in (0, 50):
+                    srng = ssd.binding.ssd_rng(23, step)
+                    path, nxt = p.ctx.accept_tree_sparse(buf.data_ptr(), idx, val, tokens, parent, mode=ssd.SSD_SAMPLING, temperature=1.0,
+                                                         top_k=top_k, rng=srng)
+                    opath, onxt, margin = ssd_oracle.accept_tree(got.astype(np.float32), dense, tokens, parent, mode=1, temperature=1.0,
+                                                                 top_k=top_k, seed=23, step=step)
+                    if (path, nxt) != (opath, onxt):
+                        assert margin < 1e-9, (label, "lists", top_k, step, margin)
+                        fragile += 1
         print("draws forgiven for a margin below 1e-9:", fragile)
         assert fragile == 0
         assert p.ctx.device_status() == 0
