@@ -30,11 +30,12 @@ constexpr int KROW = DH + 8;     // shared-memory K row stride (elements): 144 B
 constexpr int MAX_SPLITS = 4;
 constexpr int QROW = DH + 4;     // shared-memory row stride (floats) of the 16 query rows
 
-__host__ __device__ inline size_t smem_bytes(int n, int NW = NW_MAX, bool staged = false) {
+__host__ __device__ inline size_t smem_bytes(int n, int NW = NW_MAX, bool staged = false, int splits = 1) {
     // sized for the worst prefix alignment: up to 15 prefix-tail keys plus n tree keys (none when the tree's rows are read from the cache)
     const int lk_pad = staged ? 0 : (n + 15 + 15) & ~15;
     const int vrow = lk_pad + 8;
-    return (size_t)lk_pad * KROW * 2 + (size_t)DH * vrow * 2 + (size_t)NW * 16 * 66 * 4 + (size_t)16 * QROW * 4 + 16 * SSD_ANC_WORDS * 8 + 16;
+    return (size_t)lk_pad * KROW * 2 + (size_t)DH * vrow * 2 + (size_t)NW * 16 * 66 * 4 + (size_t)16 * QROW * 4 + 16 * SSD_ANC_WORDS * 8 + 16 +
+           (splits > 1 ? (size_t)splits * 16 * 66 * 4 : 0); // (key splits merged inside a cluster: one partial result per split, in the first CTA)
 }
 
 // Where an item's result goes.
@@ -43,6 +44,8 @@ struct Output {
     float *part_o;              // several splits: [split][max_nodes][d] un-normalised sums
     float *part_ml;             // several splits: [split][max_nodes][n_head][2] running max and sum
     int max_nodes, n_head;
+    int cluster_merge;          // several splits that are the CTAs of ONE thread-block cluster (split = rank): each sends its partial
+                                // result to the first CTA's shared memory, which merges them and writes the output as with one split
     uint8_t *planes8;           // one split, 8-bit projections: the output as four e4m3 planes [4][rows][d] instead of o_hi / o_lo
     size_t plane_stride;
 };
@@ -98,6 +101,7 @@ __device__ __forceinline__ void work_item(int tid, int bar_id, unsigned char *sm
     float *s_merge = reinterpret_cast<float *>(s_v + (size_t)DH * vrow);           // [NW][16][66]: m, l, o[64]
     float *s_q = s_merge + (size_t)NW * 16 * 66;                                   // [16][QROW] query rows of the tile (fp32)
     uint64_t *s_anc = reinterpret_cast<uint64_t *>(s_q + 16 * QROW);               // [16][SSD_ANC_WORDS] ancestor masks of the tile's rows
+    float *s_cl = reinterpret_cast<float *>(s_anc + 16 * SSD_ANC_WORDS);           // [n_splits][16][66] (cluster merge, used in the first CTA)
 
     const int n_blocks = (n_keys + 15) >> 4;
     const int b_lo = (n_blocks * split) / n_splits, b_hi = (n_blocks * (split + 1)) / n_splits;
@@ -341,7 +345,12 @@ __device__ __forceinline__ void work_item(int tid, int bar_id, unsigned char *sm
                 for (int q = 0; q < 4; ++q) acc[q] += src[2 + c0 + q] * wgt;
             }
             const size_t at = (size_t)row * d + h * DH + c0;
-            if (n_splits == 1) {
+            if (n_splits > 1 && out.cluster_merge) { // this split's (max, sum, un-normalised output) of the row -> the first CTA of the cluster
+                const uint32_t dst = ptx::mapa_shared(ptx::smem_u32(s_cl + ((size_t)split * 16 + r) * 66), 0);
+                if (c0 == 0) { ptx::st_cluster_f32(dst, M); ptx::st_cluster_f32(dst + 4, L); }
+#pragma unroll
+                for (int q = 0; q < 4; ++q) ptx::st_cluster_f32(dst + (2 + c0 + q) * 4, acc[q]);
+            } else if (n_splits == 1) {
                 const float inv = 1.0f / L; // a node always sees itself, so L > 0
                 if (out.planes8) { w8::store4(out.planes8, out.plane_stride, at, acc[0] * inv, acc[1] * inv, acc[2] * inv, acc[3] * inv); continue; }
                 uint32_t h0, l0, h1, l1;
@@ -353,6 +362,34 @@ __device__ __forceinline__ void work_item(int tid, int bar_id, unsigned char *sm
                 *reinterpret_cast<float4 *>(out.part_o + (size_t)split * out.max_nodes * d + at) = make_float4(acc[0], acc[1], acc[2], acc[3]);
                 if (c0 == 0)
                     *reinterpret_cast<float2 *>(out.part_ml + (((size_t)split * out.max_nodes + row) * out.n_head + h) * 2) = make_float2(M, L);
+            }
+        }
+    }
+    if (n_splits > 1 && out.cluster_merge) {
+        ptx::cluster_arrive_release();
+        ptx::cluster_wait_acquire();
+        if (split == 0) { // the same merge once more, over the splits' results
+            for (int slot = tid; slot < 256; slot += NW * 32) {
+                const int r = slot >> 4, c0 = (slot & 15) * 4, row = tile0 + r;
+                if (row >= n) continue;
+                float M = -INFINITY;
+                for (int w = 0; w < n_splits; ++w) M = fmaxf(M, s_cl[((size_t)w * 16 + r) * 66]);
+                float L = 0.f, acc[4] = {0.f, 0.f, 0.f, 0.f};
+                for (int w = 0; w < n_splits; ++w) {
+                    const float *src = s_cl + ((size_t)w * 16 + r) * 66;
+                    const float wgt = (src[0] == -INFINITY) ? 0.f : __expf(src[0] - M);
+                    L += src[1] * wgt;
+#pragma unroll
+                    for (int q = 0; q < 4; ++q) acc[q] += src[2 + c0 + q] * wgt;
+                }
+                const size_t at = (size_t)row * d + h * DH + c0;
+                const float inv = 1.0f / L; // a node always sees itself, so L > 0
+                if (out.planes8) { w8::store4(out.planes8, out.plane_stride, at, acc[0] * inv, acc[1] * inv, acc[2] * inv, acc[3] * inv); continue; }
+                uint32_t h0, l0, h1, l1;
+                split_pair(acc[0] * inv, acc[1] * inv, h0, l0);
+                split_pair(acc[2] * inv, acc[3] * inv, h1, l1);
+                *reinterpret_cast<uint2 *>(out.o_hi + at) = make_uint2(h0, h1);
+                if (out.o_lo) *reinterpret_cast<uint2 *>(out.o_lo + at) = make_uint2(l0, l1);
             }
         }
     }

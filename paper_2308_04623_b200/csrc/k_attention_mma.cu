@@ -55,10 +55,14 @@ tree_attention_mma_kernel(const float *__restrict__ qkv, const StepInfo *__restr
     extern __shared__ __align__(16) unsigned char smem_raw[];
     if (threadIdx.x == 0) ptx::trace_mark(trace, 0);
     ptx::pdl_launch_dependents();
-    attn::Output out = {o_hi, o_lo, nullptr, nullptr, 0, 0, planes8, plane_stride};
+    // Long prefixes: gridDim.z CTAs - one thread-block cluster - share a (head, node tile), each with a contiguous part of the key
+    // blocks; the last one holds the tree's own keys (and, for tile 0, writes them to the cache's scratch slots).
+    const int splits = gridDim.z, split = blockIdx.z;
+    attn::Output out = {o_hi, o_lo, nullptr, nullptr, 0, 0, splits > 1 ? 1 : 0, planes8, plane_stride};
     // (the step's tree metadata and the committed cache rows were complete before the first dependent launch of the
     //  forward began, so the item reads them before it waits for the QKV projection)
-    attn::work_item<(STAGED ? NW_STAGED : attn::NW_MAX), true, true, LO, STAGED>(threadIdx.x, 0, smem_raw, blockIdx.x, blockIdx.y * 16, 0, 1, blockIdx.y == 0, qkv, info, layer_offset, meta, n, d, cap, out, trace);
+    attn::work_item<(STAGED ? NW_STAGED : attn::NW_MAX), true, true, LO, STAGED>(threadIdx.x, 0, smem_raw, blockIdx.x, blockIdx.y * 16, split, splits,
+                                                                                 blockIdx.y == 0 && split == splits - 1, qkv, info, layer_offset, meta, n, d, cap, out, trace);
     if (trace) { __syncthreads(); if (threadIdx.x == 0) ptx::trace_mark(trace, 2); }
 }
 } // namespace
@@ -70,7 +74,7 @@ cudaError_t tree_attention_mma_prepare() {
     const void *kernels[] = {(const void *)tree_attention_mma_kernel<true, false>, (const void *)tree_attention_mma_kernel<false, false>,
                              (const void *)tree_attention_mma_kernel<true, true>, (const void *)tree_attention_mma_kernel<false, true>};
     for (const void *k : kernels) {
-        if (e == cudaSuccess) e = cudaFuncSetAttribute(k, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)tree_attention_mma_smem(SSD_MAX_NODES));
+        if (e == cudaSuccess) e = cudaFuncSetAttribute(k, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)attn::smem_bytes(SSD_MAX_NODES, attn::NW_MAX, false, 8));
         if (e == cudaSuccess) e = cudaFuncSetAttribute(k, cudaFuncAttributePreferredSharedMemoryCarveout, cudaSharedmemCarveoutMaxShared);
     }
     if (e == cudaSuccess) e = cudaFuncSetAttribute(kv_stage_kernel, cudaFuncAttributePreferredSharedMemoryCarveout, cudaSharedmemCarveoutMaxShared);
@@ -93,17 +97,27 @@ cudaError_t launch_kv_stage(const float *qkv, const StepInfo *info, size_t layer
 
 cudaError_t launch_tree_attention_mma(const float *qkv, const StepInfo *info, size_t layer_offset_elems, const TreeMeta &m, int n, int n_head,
                                       int cap, __nv_bfloat16 *o_hi, __nv_bfloat16 *o_lo, bool pdl, cudaStream_t s, unsigned long long *trace, bool lo_pairs,
-                                      uint8_t *planes8, size_t plane_stride, bool staged) {
+                                      uint8_t *planes8, size_t plane_stride, bool staged, int splits) {
+    if (splits < 1 || splits > 8 || (staged && splits != 1)) return cudaErrorInvalidValue;
     cudaLaunchConfig_t cfg = {};
-    cfg.gridDim = dim3(n_head, (n + 15) / 16);
+    cfg.gridDim = dim3(n_head, (n + 15) / 16, splits);
     cfg.blockDim = dim3((staged ? NW_STAGED : attn::NW_MAX) * 32);
-    cfg.dynamicSmemBytes = attn::smem_bytes(n, staged ? NW_STAGED : attn::NW_MAX, staged);
+    cfg.dynamicSmemBytes = attn::smem_bytes(n, staged ? NW_STAGED : attn::NW_MAX, staged, splits);
     cfg.stream = s;
-    cudaLaunchAttribute attr[1];
-    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
-    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cudaLaunchAttribute attr[2];
+    int na = 0;
+    if (pdl) {
+        attr[na].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+        attr[na].val.programmaticStreamSerializationAllowed = 1;
+        ++na;
+    }
+    if (splits > 1) {
+        attr[na].id = cudaLaunchAttributeClusterDimension;
+        attr[na].val.clusterDim.x = 1; attr[na].val.clusterDim.y = 1; attr[na].val.clusterDim.z = (unsigned)splits;
+        ++na;
+    }
     cfg.attrs = attr;
-    cfg.numAttrs = pdl ? 1 : 0;
+    cfg.numAttrs = na;
     auto kernel = staged ? (lo_pairs ? tree_attention_mma_kernel<true, true> : tree_attention_mma_kernel<false, true>)
                          : (lo_pairs ? tree_attention_mma_kernel<true, false> : tree_attention_mma_kernel<false, false>);
     return cudaLaunchKernelEx(&cfg, kernel, qkv, info, layer_offset_elems, m, n, n_head * attn::DH, cap, o_hi, o_lo, trace, planes8, plane_stride);

@@ -103,6 +103,26 @@ __device__ __forceinline__ uint64_t policy_evict_first() {
     return p;
 }
 
+// ---- thread-block clusters: another CTA's shared memory ----------------------------------------
+__device__ __forceinline__ uint32_t cluster_ctarank() {
+    uint32_t r;
+    asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r));
+    return r;
+}
+// The address, in the cluster's shared window, of `smem_addr` (an address of this CTA's shared memory) in CTA `rank`.
+__device__ __forceinline__ uint32_t mapa_shared(uint32_t smem_addr, uint32_t rank) {
+    uint32_t r;
+    asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"(smem_addr), "r"(rank));
+    return r;
+}
+__device__ __forceinline__ void st_cluster_f32(uint32_t cluster_addr, float v) {
+    asm volatile("st.shared::cluster.f32 [%0], %1;" ::"r"(cluster_addr), "f"(v) : "memory");
+}
+// Cluster-wide barrier that also orders memory: what a CTA wrote (into a peer's shared memory too) before arriving is
+// visible to every CTA after its wait.  Every thread of every CTA of the cluster executes both.
+__device__ __forceinline__ void cluster_arrive_release() { asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory"); }
+__device__ __forceinline__ void cluster_wait_acquire() { asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory"); }
+
 // ---- tcgen05 / TMEM ----------------------------------------------------------------------
 // Allocation is a warp-wide (.sync.aligned) operation; the base address lands in shared memory.
 __device__ __forceinline__ void tmem_alloc(uint32_t *smem_result, uint32_t ncols) {

@@ -62,7 +62,8 @@ struct ssd_ctx {
     // step (prefix length, cache and output addresses) from d_info, and the tree itself travels
     // in the arguments of the first node, which are patched before each launch.
     struct ForwardGraph { cudaGraph_t graph; cudaGraphExec_t exec; cudaGraphNode_t prep_node; int kernels; };
-    ForwardGraph graphs[SSD_MAX_NODES + 1];
+    ForwardGraph graphs[SSD_MAX_NODES + 1][3]; // (second index: the attention's key splits, 1 / 2 / 4 - chosen from the prefix length at each call)
+    int attn_splits;                           // 0 = choose; 1, 2, 4 = always that many
     cudaStream_t capture_stream;
     AcceptScratch acc;
     int32_t *h_result; // pinned host copy of acc.result
@@ -213,8 +214,24 @@ static unsigned long long *trace_slot(ssd_ctx *ctx, int kernels) {
 }
 
 // Enqueue every kernel of one tree-batched forward on `s`.
+// Key splits of the attention for a step: a warp should have about two 16-key blocks; more CTAs per (head, node tile) only while
+// they all fit the GPU at once, and not on the large-tree path.  Measured (verify, us): GPT-2-small shape, prefix 512, 8 nodes:
+// 322 / 309 / 302 with 1 / 2 / 4 splits; GPT-2-XL shape, prefix 960, 8 nodes: 1993 / 1864 / 1705; prefix 512, 32 nodes: 1799 / 1763 /
+// 1979 (200 CTAs: two waves); GPT-2-large shape, prefix 256, 32 nodes (18 key blocks): 1057 / 1096.
+static int attn_splits_for(const ssd_ctx *ctx, int kv_len, int n) {
+    const int tiles = (n + 15) / 16, ctas = ctx->cfg.n_head * tiles;
+    const bool staged = ctx->stage_kv_from > 0 && n >= ctx->stage_kv_from;
+    int s = ctx->attn_splits;
+    if (s == 0) {
+        const int blocks = (kv_len + n + 15) / 16;
+        s = blocks > 54 ? 4 : blocks > 27 ? 2 : 1;
+    }
+    while (s > 1 && (staged || ctas * s > ctx->sm_count)) s >>= 1; // (an attention CTA has an SM to itself: more CTAs than SMs run in waves)
+    return s;
+}
+
 cudaError_t enqueue_forward(ssd_ctx *ctx, int n, int cap, const NodeList &tk, const NodeList &pr, const StepInfo &step, cudaStream_t s,
-                            int *kernels) {
+                            int *kernels, int attn_splits = 1) {
     const ssd_config &c = ctx->cfg;
     const int d = c.d_model, F = c.d_ff, max_keys = c.n_ctx + n;
     const size_t layer_elems = (size_t)c.n_head * cap * 64;
@@ -311,7 +328,7 @@ cudaError_t enqueue_forward(ssd_ctx *ctx, int n, int cap, const NodeList &tk, co
                 Q(launch_ln_prep(ctx->x, L.ln1_g, L.ln1_b, n, d, c.ln_eps, nullptr, nullptr, ctx->qkv, 3 * d, info, 0, pdl, s, trace_slot(ctx, *kernels), ctx->a8, sa));
                 Q(gemm8(&t[0], &ssd_ctx::ActMaps::a_hi, ctx->qkv, 3 * d, L.b_qkv, d, 3 * d, grid, L.s_qkv));
                 if (staged) Q(launch_kv_stage(ctx->qkv, info, l * layer_elems, n, c.n_head, cap, pdl, s, trace_slot(ctx, *kernels)));
-                Q(launch_tree_attention_mma(ctx->qkv, info, l * layer_elems, ctx->meta, n, c.n_head, cap, nullptr, nullptr, pdl, s, trace_slot(ctx, *kernels), ctx->attn_lo != 0, ctx->o8, sa, staged));
+                Q(launch_tree_attention_mma(ctx->qkv, info, l * layer_elems, ctx->meta, n, c.n_head, cap, nullptr, nullptr, pdl, s, trace_slot(ctx, *kernels), ctx->attn_lo != 0, ctx->o8, sa, staged, attn_splits));
                 Q(gemm8(&t[1], &ssd_ctx::ActMaps::o_hi, ctx->x, d, L.b_o, d, d, grid, L.s_o));
                 Q(launch_ln_prep(ctx->x, L.ln2_g, L.ln2_b, n, d, c.ln_eps, nullptr, nullptr, ctx->h, F, info, 0, pdl, s, trace_slot(ctx, *kernels), ctx->a8, sa));
                 Q(gemm8(&t[2], &ssd_ctx::ActMaps::a_hi, ctx->h, F, L.b_fc, d, F, grid, L.s_fc));
@@ -329,7 +346,7 @@ cudaError_t enqueue_forward(ssd_ctx *ctx, int n, int cap, const NodeList &tk, co
             Q(launch_ln_prep(ctx->x, L.ln1_g, L.ln1_b, n, d, c.ln_eps, ctx->a_hi, a_lo, ctx->qkv, 3 * d, info, 0, pdl, s, trace_slot(ctx, *kernels)));
             Q(launch_gemm_ws(&t[0], &am->a_hi, &am->a_pair, ctx->qkv, info, 3 * d, L.b_qkv, n, d, 3 * d, lo, grid, sms, ctx->d_status, pdl, s, trace_slot(ctx, *kernels)));
             if (staged) Q(launch_kv_stage(ctx->qkv, info, l * layer_elems, n, c.n_head, cap, pdl, s, trace_slot(ctx, *kernels)));
-            Q(launch_tree_attention_mma(ctx->qkv, info, l * layer_elems, ctx->meta, n, c.n_head, cap, ctx->o_hi, o_lo, pdl, s, trace_slot(ctx, *kernels), ctx->attn_lo != 0, nullptr, 0, staged));
+            Q(launch_tree_attention_mma(ctx->qkv, info, l * layer_elems, ctx->meta, n, c.n_head, cap, ctx->o_hi, o_lo, pdl, s, trace_slot(ctx, *kernels), ctx->attn_lo != 0, nullptr, 0, staged, attn_splits));
             Q(launch_gemm_ws(&t[1], &am->o_hi, &am->o_pair, ctx->x, info, d, L.b_o, n, d, d, lo, grid, sms, ctx->d_status, pdl, s, trace_slot(ctx, *kernels)));
             Q(launch_ln_prep(ctx->x, L.ln2_g, L.ln2_b, n, d, c.ln_eps, ctx->a_hi, a_lo, ctx->h, F, info, 0, pdl, s, trace_slot(ctx, *kernels)));
             Q(launch_gemm_ws(&t[2], &am->a_hi, &am->a_pair, ctx->h, info, F, L.b_fc, n, d, F, lo, grid, sms, ctx->d_status, pdl, s, trace_slot(ctx, *kernels)));
@@ -358,12 +375,12 @@ cudaError_t enqueue_forward(ssd_ctx *ctx, int n, int cap, const NodeList &tk, co
 }
 
 // Capture the forward for tree size n into an executable graph and remember its first node.
-int capture_forward(ssd_ctx *ctx, int n, int cap, const NodeList &tk, const NodeList &pr, const StepInfo &step) {
-    ssd_ctx::ForwardGraph &fg = ctx->graphs[n];
+int capture_forward(ssd_ctx *ctx, int n, int cap, const NodeList &tk, const NodeList &pr, const StepInfo &step, int attn_splits) {
+    ssd_ctx::ForwardGraph &fg = ctx->graphs[n][attn_splits >> 1];
     cudaGraph_t graph = nullptr;
     int kernels = 0;
     CU(cudaStreamBeginCapture(ctx->capture_stream, cudaStreamCaptureModeThreadLocal));
-    cudaError_t e = enqueue_forward(ctx, n, cap, tk, pr, step, ctx->capture_stream, &kernels);
+    cudaError_t e = enqueue_forward(ctx, n, cap, tk, pr, step, ctx->capture_stream, &kernels, attn_splits);
     cudaError_t e2 = cudaStreamEndCapture(ctx->capture_stream, &graph);
     if (e != cudaSuccess || e2 != cudaSuccess) {
         if (graph) cudaGraphDestroy(graph);
@@ -456,6 +473,7 @@ int ssd_create(const ssd_config *cfg, int device, void *cuda_stream, ssd_ctx **o
     if (ctx->w8) ctx->cfg.dtype = SSD_DTYPE_BF16;
     ctx->wte8 = nullptr; ctx->wte_scale = nullptr;
     ctx->w8_planes = 4;
+    ctx->attn_splits = 0;
     ctx->stage_kv_from = 128; // (measured at the GPT-2-large shape: 2 % faster at 128 nodes, 14 % at 256, slower below)
     ctx->device = device;
     ctx->stream = (cudaStream_t)cuda_stream;
@@ -553,8 +571,9 @@ void ssd_destroy(ssd_ctx *ctx) {
     if (!ctx) return;
     DeviceGuard g(ctx->device);
     cudaStreamSynchronize(ctx->stream);
-    for (auto &g : ctx->graphs)
-        if (g.exec) { cudaGraphExecDestroy(g.exec); cudaGraphDestroy(g.graph); }
+    for (auto &row : ctx->graphs)
+        for (auto &g : row)
+            if (g.exec) { cudaGraphExecDestroy(g.exec); cudaGraphDestroy(g.graph); }
     if (ctx->capture_stream) cudaStreamDestroy(ctx->capture_stream);
     for (void *p : ctx->owned) cudaFree(p);
     if (ctx->acc.rows) cudaFree(ctx->acc.rows);
@@ -762,10 +781,11 @@ int ssd_verify_tree(ssd_ctx *ctx, const int32_t *tokens, const int32_t *parent_i
     StepInfo step;
     step.n = n_nodes; step.kv_len = kv->len; step.kbase = kv->k; step.vbase = kv->v; step.logits = logits_out;
     int kernels = 0;
+    const int splits = ctx->tensor_path ? attn_splits_for(ctx, kv->len, n_nodes) : 1;
     if (ctx->tensor_path && ctx->use_graph) {
-        ssd_ctx::ForwardGraph &fg = ctx->graphs[n_nodes];
+        ssd_ctx::ForwardGraph &fg = ctx->graphs[n_nodes][splits >> 1];
         if (!fg.exec) {
-            rc = capture_forward(ctx, n_nodes, kv->cap, tk, pr, step);
+            rc = capture_forward(ctx, n_nodes, kv->cap, tk, pr, step, splits);
             if (rc != SSD_OK) return rc;
         }
         // patch the tree, prefix length and addresses into the first node, then replay
@@ -779,7 +799,7 @@ int ssd_verify_tree(ssd_ctx *ctx, const int32_t *tokens, const int32_t *parent_i
         CU(cudaGraphLaunch(fg.exec, ctx->stream));
         kernels = fg.kernels;
     } else {
-        CU(enqueue_forward(ctx, n_nodes, kv->cap, tk, pr, step, ctx->stream, &kernels));
+        CU(enqueue_forward(ctx, n_nodes, kv->cap, tk, pr, step, ctx->stream, &kernels, splits));
     }
     ctx->launches += kernels;
     ctx->head_logits = (ctx->tensor_path && ctx->use_head_stats) ? logits_out : nullptr;
@@ -986,6 +1006,7 @@ int ssd_set_tuning(ssd_ctx *ctx, int32_t knob, int32_t value) {
     case SSD_TUNE_ATTN_LOW_PLANE: if (value != 0 && value != 1) return SSD_ERR_BAD_ARG; ctx->attn_lo = value; break;
     case SSD_TUNE_HEAD_STATS: if (value != 0 && value != 1) return SSD_ERR_BAD_ARG; ctx->use_head_stats = value; ctx->head_logits = nullptr; break;
     case SSD_TUNE_STAGE_KV_FROM: if (value < 0 || value > SSD_MAX_NODES + 1) return SSD_ERR_BAD_ARG; ctx->stage_kv_from = value; break;
+    case SSD_TUNE_ATTN_SPLITS: if (value != 0 && value != 1 && value != 2 && value != 4) return SSD_ERR_BAD_ARG; ctx->attn_splits = value; break;
     case SSD_TUNE_W8_PLANES:
         if (!ctx->w8 || value < 2 || value > 4) return SSD_ERR_BAD_ARG;
         ctx->w8_planes = value;
@@ -1000,8 +1021,9 @@ int ssd_set_tuning(ssd_ctx *ctx, int32_t knob, int32_t value) {
     DeviceGuard g(ctx->device);
     if (!g.ok) return SSD_ERR_CUDA;
     CU(cudaStreamSynchronize(ctx->stream));
-    for (auto &fg : ctx->graphs) // captured forwards bake the old setting in
-        if (fg.exec) { cudaGraphExecDestroy(fg.exec); cudaGraphDestroy(fg.graph); fg.exec = nullptr; fg.graph = nullptr; }
+    for (auto &row : ctx->graphs) // captured forwards bake the old setting in
+        for (auto &fg : row)
+            if (fg.exec) { cudaGraphExecDestroy(fg.exec); cudaGraphDestroy(fg.graph); fg.exec = nullptr; fg.graph = nullptr; }
     return SSD_OK;
 }
 int ssd_get_phase_trace(ssd_ctx *ctx, uint64_t *out_ns, int32_t capacity, int32_t *count) {

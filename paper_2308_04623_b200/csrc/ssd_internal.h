@@ -139,13 +139,15 @@ cudaError_t launch_kv_commit(void *kbase, void *vbase, int dtype, int n_layer, i
                              int n_path, cudaStream_t s, int *launches);
 cudaError_t launch_kv_read(const void *cache_layer, int dtype, int n_head, int cap, int slot0, int rows, int transposed, float *out,
                            cudaStream_t s);
+// (splits > 1: that many CTAs - one thread-block cluster - share a (head, node tile), each taking a part of the key blocks; their
+//  partial softmaxes are merged in the first one's shared memory.  Worth it for long prefixes.)
 // bf16 path attention on mma.sync tiles; K cache [H, cap, 64], V cache transposed [H, 64, cap]; cap a multiple of 16.
 size_t tree_attention_mma_smem(int n);
 cudaError_t tree_attention_mma_prepare();
 cudaError_t launch_tree_attention_mma(const float *qkv, const StepInfo *info, size_t layer_offset_elems, const TreeMeta &m, int n, int n_head,
                                       int cap, __nv_bfloat16 *o_hi, __nv_bfloat16 *o_lo, bool pdl, cudaStream_t s,
                                       unsigned long long *trace = nullptr, bool lo_pairs = true, uint8_t *planes8 = nullptr,
-                                      size_t plane_stride = 0, bool staged = false);
+                                      size_t plane_stride = 0, bool staged = false, int splits = 1);
 // Writes the tree's K / V rows (bf16) to the cache's scratch slots and zeroes the rest of the last 16-key block; an attention launched
 // with `staged` then reads every block from the cache and stages nothing itself (worth its launch for large trees).
 cudaError_t launch_kv_stage(const float *qkv, const StepInfo *info, size_t layer_offset_elems, int n, int n_head, int cap, bool pdl, cudaStream_t s,

@@ -865,3 +865,41 @@ def test_tree_rows_read_from_the_cache_give_the_same_logits(ssd, util, prefix):
         p.commit(path)
     assert p.ctx.device_status() == 0
     p.close()
+
+
+@pytest.mark.parametrize("splits", [2, 4])
+def test_attention_key_splits_merged_in_a_cluster(ssd, util, splits):
+    """Several CTAs - one thread-block cluster - share a (head, node tile), each with a part of the key blocks, merged in the first
+    one's shared memory.  Forced on short prefixes too (some splits then hold no block at all, or only masked keys) and compared with
+    the oracle and with the single-CTA path; commits in between check that the tree's K / V rows still reach the cache (the
+    last split of tile 0 writes them); then with the split count chosen from the prefix length."""
+    rng = np.random.default_rng(71 + splits)
+    p = util.Pair("ragged_bf16", seed=5, qk_gain=3.0)
+    V, L = p.V, p.cfg["n_layer"]
+    for prefix_add, n in ((0, 1), (3, 9), (13, 40), (16, 64), (60, 21), (90, 100)):
+        par = ssd_synth.tree_random(n, 6, rng)
+        tok = ssd_synth.uniform_tokens(n, V, rng)
+        p.ctx.set_tuning(ssd.SSD_TUNE_ATTN_SPLITS, splits)
+        got, want, _ = p.verify(tok, par)
+        p.ctx.set_tuning(ssd.SSD_TUNE_ATTN_SPLITS, 1)
+        plain, _, _ = p.verify(tok, par)
+        assert np.isfinite(got).all()
+        assert np.abs(got - want).max() <= TOL_BF16, (splits, n)
+        assert np.abs(got - plain).max() <= 2e-3, (splits, n)
+        p.ctx.set_tuning(ssd.SSD_TUNE_ATTN_SPLITS, splits)
+        got2, _, _ = p.verify(tok, par)                      # (the scratch rows the commit below moves come from this forward)
+        path = ssd_synth.path_to(par, int(rng.integers(0, n)))
+        p.commit(path)
+        extra = int(prefix_add)
+        for _ in range(extra):                                  # grow the prefix one committed root at a time, splits still forced
+            t1 = ssd_synth.uniform_tokens(1, V, rng)
+            p.verify(t1, np.array([-1], dtype=np.int32))
+            p.commit([0])
+    p.ctx.set_tuning(ssd.SSD_TUNE_ATTN_SPLITS, 0)
+    assert len(p.kv) > 150                                      # long enough for the automatic choice to split
+    par = ssd_synth.tree_random(12, 5, rng)
+    tok = ssd_synth.uniform_tokens(12, V, rng)
+    got, want, _ = p.verify(tok, par)
+    assert np.abs(got - want).max() <= TOL_BF16
+    assert p.ctx.device_status() == 0
+    p.close()
