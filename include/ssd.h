@@ -282,11 +282,13 @@ int ssd_kv_read(ssd_ctx *ctx, const ssd_kv *kv, int32_t layer, int32_t which, in
  *   SSD_TUNE_ATTN_SPLITS [0]      bf16 models: CTAs (one thread-block cluster) that share a (head, 16-node tile) of the attention, each
  *                                 with a part of the keys, merged in the first one's shared memory: 1, 2 or 4; 0 = from the prefix
  *                                 length of each call (1 up to 27 key blocks of 16, 2 up to 54, else 4)
+ *   SSD_TUNE_NODE_GROUPS [1]      bf16 models, trees of more than 128 nodes: the layers' projections run on node groups of 64 (one
+ *                                 copy of a 64-node tree's CTA arrangement per group) instead of on the whole batch per CTA
  *   SSD_TUNE_KERNEL_TRACE [0]     record a timeline of every kernel of a bf16 forward (see ssd_get_phase_trace)
  */
 enum { SSD_TUNE_LOW_PLANE = 0, SSD_TUNE_DEPENDENT_LAUNCH = 1, SSD_TUNE_GRAPH = 2, SSD_TUNE_GEMM_CTAS = 3, SSD_TUNE_CLUSTER_REDUCE = 4,
        SSD_TUNE_CLUSTER_MAX = 5, SSD_TUNE_ATTN_LOW_PLANE = 6, SSD_TUNE_HEAD_CTAS = 7, SSD_TUNE_KERNEL_TRACE = 8, SSD_TUNE_CLUSTER_QKV = 9, SSD_TUNE_CLUSTER_O = 10,
-       SSD_TUNE_CLUSTER_FC = 11, SSD_TUNE_CLUSTER_PROJ = 12, SSD_TUNE_HEAD_STATS = 13, SSD_TUNE_W8_PLANES = 14, SSD_TUNE_STAGE_KV_FROM = 15, SSD_TUNE_ATTN_SPLITS = 16 };
+       SSD_TUNE_CLUSTER_FC = 11, SSD_TUNE_CLUSTER_PROJ = 12, SSD_TUNE_HEAD_STATS = 13, SSD_TUNE_W8_PLANES = 14, SSD_TUNE_STAGE_KV_FROM = 15, SSD_TUNE_ATTN_SPLITS = 16, SSD_TUNE_NODE_GROUPS = 17 };
 int ssd_set_tuning(ssd_ctx *ctx, int32_t knob, int32_t value);
 
 /*

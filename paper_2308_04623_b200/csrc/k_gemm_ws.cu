@@ -35,6 +35,12 @@
 //     instruction multiplies a weight slice by all four (N = 4 n_pad <= 256; two instructions for 128 rows), each
 //     plane's product in accumulator columns of its own.  The epilogue adds the four with their powers of two and
 //     multiplies by the row's scale.  At most 128 rows per launch (512 accumulator columns).
+//   * large trees: the nodes are cut into GROUPS of 64 and the grid is `groups` copies of the CTA arrangement of a
+//     64-node tree, copy g working on nodes 64 g .. 64 g + 63 (its activation boxes start at that row, its sums go
+//     to those rows of Y).  The weights are not read more often for it - the copies run at the same time and the
+//     tile one of them fetches is in L2 for the others - but what grows with the tree no longer lands on one CTA:
+//     one instruction still covers hi and lo (N = 128), two CTAs still share an SM, the epilogue drains 64 nodes,
+//     not 256, and with the CTAs spread over node groups a tile's K needs fewer splits, hence fewer partial sums.
 #include <cuda.h>
 #include <cstring>
 
@@ -70,6 +76,7 @@ struct GemmParams {
     const float *w_scale; // W8: [out] scale of each output row's codes
     int planes;        // W8: how many of the four e4m3 planes of the activations take part (2..4)
     int row0;          // first activation row (node) of this launch (W8 with more than 128 nodes runs in two launches)
+    int groups;        // node groups (1 = the whole batch); group g = CTAs [g * gridDim.x / groups, ...) on nodes g * n_pad .. (n = ALL nodes then)
     // LM head with complete sums (split == 1): plain stores instead of reductions, and per (row, output tile) the maximum,
     // its lowest index and a non-finite flag, so that greedy acceptance need not read the logits again
     int store;
@@ -112,16 +119,19 @@ gemm_ws_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant_
     Barriers *bars = reinterpret_cast<Barriers *>(smem + (size_t)p.stages * stage_bytes);
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    // node group of this CTA, its index among the group's CTAs, the group's rows
+    const int cpg = gridDim.x / p.groups, grp = blockIdx.x / cpg, bid = blockIdx.x - grp * cpg;
+    const int row0 = p.row0 + grp * p.n_pad, n_rows = p.groups > 1 ? min(p.n_pad, p.n - grp * p.n_pad) : p.n;
     // this CTA's contiguous range of (tile, k tile) units
     const long long units = (long long)p.n_tiles * p.k_tiles;
     int u0, u1;
     if (p.split > 0) { // tile-aligned: no CTA straddles two output tiles, so each runs exactly one epilogue
-        const int tile = blockIdx.x / p.split, r = blockIdx.x - tile * p.split;
+        const int tile = bid / p.split, r = bid - tile * p.split;
         u0 = tile * p.k_tiles + (p.k_tiles * r) / p.split;
         u1 = tile * p.k_tiles + (p.k_tiles * (r + 1)) / p.split;
     } else {
-        u0 = (int)((units * blockIdx.x) / gridDim.x);
-        u1 = (int)((units * (blockIdx.x + 1)) / gridDim.x);
+        u0 = (int)((units * bid) / cpg);
+        u1 = (int)((units * (bid + 1)) / cpg);
     }
     // The hi and lo planes of the activations are adjacent in a stage, so while 2 * n_pad <= 256 ONE MMA
     // covers both (N = 2 * n_pad, the lo part lands in its own accumulator columns and is added in the
@@ -197,12 +207,12 @@ gemm_ws_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant_
                 }
                 // (the activation maps' box is the whole padded batch: one operation per plane; W8: one for the four planes)
                 if (W8) {
-                    ptx::tma_load_3d(st + A_BYTES, &map_hi, kt * KT, p.row0, 0, &bars->full[s]);
+                    ptx::tma_load_3d(st + A_BYTES, &map_hi, kt * KT, row0, 0, &bars->full[s]);
                 } else {
                     // (with the lo plane: ONE box over both planes - they are adjacent in memory as in the stage - since every copy
                     //  this one thread issues costs it some 50-100 ns ahead of the first MMA)
-                    if (p.use_lo) ptx::tma_load_3d(st + A_BYTES, &map_lo, kt * TILE_K, 0, 0, &bars->full[s]);
-                    else ptx::tma_load_2d(st + A_BYTES, &map_hi, kt * TILE_K, 0, &bars->full[s]);
+                    if (p.use_lo) ptx::tma_load_3d(st + A_BYTES, &map_lo, kt * TILE_K, row0, 0, &bars->full[s]);
+                    else ptx::tma_load_2d(st + A_BYTES, &map_hi, kt * TILE_K, row0, &bars->full[s]);
                 }
                 if (bars->abort) ok = false;
                 if (++kt == p.k_tiles) { kt = 0; ++tile; }
@@ -292,8 +302,8 @@ gemm_ws_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant_
                     if (p.planes > 3) ptx::tmem_ld_32x16(taddr + 3 * p.n_pad + c0, a3);
                     ptx::tmem_ld_wait();
                     if (o < p.out) {
-                        float *yo = y + (size_t)(p.row0 + c0) * p.ldy + o;
-                        const int rows = min(16, p.n - c0);
+                        float *yo = y + (size_t)(row0 + c0) * p.ldy + o;
+                        const int rows = min(16, n_rows - c0);
 #pragma unroll
                         for (int t = 0; t < 16; ++t, yo += p.ldy) {
                             const float hi = fmaf(16.f, __uint_as_float(a0[t]), __uint_as_float(a1[t]));
@@ -314,7 +324,7 @@ gemm_ws_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant_
 #pragma unroll
                     for (int t = 0; t < 16; ++t) {
                         v[t] = __uint_as_float(r[t]) + (stacked ? __uint_as_float(q[t]) : 0.f) + bias;
-                        if (o < p.out && c0 + t < p.n) y[(size_t)(c0 + t) * p.ldy + o] = v[t];
+                        if (o < p.out && c0 + t < n_rows) y[(size_t)(row0 + c0 + t) * p.ldy + o] = v[t];
                     }
                     if (p.stat_val) {
                         // row maximum over this warp's 32 features with one warp-wide integer reduction per row: floats map to
@@ -322,28 +332,28 @@ gemm_ws_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant_
 #pragma unroll
                         for (int t = 0; t < 16; ++t) {
                             const bool live = o < p.out;
-                            warp_bad |= (live && c0 + t < p.n && !isfinite(v[t])) ? 1 : 0;
+                            warp_bad |= (live && c0 + t < n_rows && !isfinite(v[t])) ? 1 : 0;
                             const unsigned bits = __float_as_uint(v[t]);
                             unsigned key = (bits & 0x80000000u) ? ~bits : (bits | 0x80000000u);
                             if (!live || v[t] != v[t]) key = 0u;       // (padding features and NaNs never win; the flag reports NaNs)
                             const unsigned top = __reduce_max_sync(0xffffffffu, key);
                             const unsigned who = __ballot_sync(0xffffffffu, key == top);
-                            if (lane == 0 && c0 + t < p.n) {
+                            if (lane == 0 && c0 + t < n_rows) {
                                 bars->stat_val[quarter][c0 + t] = top == 0u ? -INFINITY : __uint_as_float((top & 0x80000000u) ? (top & 0x7fffffffu) : ~top);
                                 bars->stat_arg[quarter][c0 + t] = tile * TILE_M + quarter * 32 + (__ffs(who) - 1);
                             }
                         }
                     }
                 } else if (o < p.out) {
-                    float *yo = y + (size_t)c0 * p.ldy + o;
-                    if (stacked && c0 + 16 <= p.n) { // the usual case, kept short: sixteen full rows, hi + lo columns
+                    float *yo = y + (size_t)(row0 + c0) * p.ldy + o;
+                    if (stacked && c0 + 16 <= n_rows) { // the usual case, kept short: sixteen full rows, hi + lo columns
 #pragma unroll
                         for (int t = 0; t < 16; ++t, yo += p.ldy) ptx::red_add_f32(yo, __uint_as_float(r[t]) + __uint_as_float(q[t]) + bias);
                     } else {
 #pragma unroll
                         for (int t = 0; t < 16; ++t) {
                             const int i = c0 + t;
-                            if (i < p.n) {
+                            if (i < n_rows) {
                                 float v = __uint_as_float(r[t]) + (stacked ? __uint_as_float(q[t]) : 0.f) + bias;
                                 ptx::red_add_f32(yo + (size_t)t * p.ldy, v);
                             }
@@ -476,12 +486,17 @@ cudaError_t gemm_ws_prepare() {
 
 cudaError_t launch_gemm_ws(const void *map_w, const void *map_hi, const void *map_lo, float *y, const StepInfo *info, int ldy,
                            const float *bias, int n, int K, int out, int use_lo, int grid, int sm_count, int32_t *status, bool pdl,
-                           cudaStream_t s, unsigned long long *trace, const GemmHeadStats *head, const float *w_scale, int row0, int w8_planes) {
+                           cudaStream_t s, unsigned long long *trace, const GemmHeadStats *head, const float *w_scale, int row0, int w8_planes, int group_rows) {
     const bool w8 = w_scale != nullptr; // map_w: the codes; map_hi: the four activation planes
     if (w8 && (n > 128 || head || w8_planes < 2 || w8_planes > W8_PLANES)) return cudaErrorInvalidValue;
+    // node groups: the activation maps' boxes hold group_rows rows (a multiple of 16), fewer than the tree has nodes
+    const bool grouped = group_rows > 0 && group_rows < n;
+    if (grouped && (w8 || head || (group_rows & 15) || row0 != 0)) return cudaErrorInvalidValue;
     GemmParams p;
     p.trace = trace;
-    p.y = y; p.info = info; p.bias = bias; p.n = n; p.n_pad = (n + 15) & ~15;
+    p.y = y; p.info = info; p.bias = bias; p.n = n; p.n_pad = grouped ? group_rows : (n + 15) & ~15;
+    p.groups = grouped ? (n + group_rows - 1) / group_rows : 1;
+    if (grouped) grid = grid / p.groups > 0 ? grid / p.groups : 1; // (the CTA count asked for is the whole launch's)
     p.out = out; p.ldy = ldy; p.k_tiles = w8 ? (K + 2 * TILE_K - 1) / (2 * TILE_K) : K / TILE_K; p.n_tiles = (out + TILE_M - 1) / TILE_M;
     p.use_lo = use_lo; p.status = status; p.w_scale = w_scale; p.row0 = row0; p.planes = w8_planes;
     p.store = 0; p.stat_val = nullptr; p.stat_arg = nullptr; p.stat_bad = nullptr;
@@ -507,14 +522,14 @@ cudaError_t launch_gemm_ws(const void *map_w, const void *map_hi, const void *ma
         p.split = 1; grid = p.n_tiles; per_cta = p.k_tiles;
         p.store = 1; p.stat_val = head->val; p.stat_arg = head->arg; p.stat_bad = head->bad;
     }
-    p.stages = gemm_ws_stages(p.n_pad, planes, grid > sm_count);
+    p.stages = gemm_ws_stages(p.n_pad, planes, grid * p.groups > sm_count);
     if (p.stages > per_cta) p.stages = per_cta < 1 ? 1 : per_cta;
     size_t smem = (size_t)p.stages * stage_bytes + sizeof(Barriers) + 1024;
     // Two CTAs per SM, not three: with a third one resident the slowest CTA of a projection ends later (measured: 1.19 ms per
     // GPT-2-large verification of 32 nodes against 1.09 ms), so a CTA asks for more than a third of an SM's shared memory.
-    if (grid > sm_count && smem < 78 * 1024) smem = 78 * 1024;
+    if (grid * p.groups > sm_count && smem < 78 * 1024) smem = 78 * 1024;
     cudaLaunchConfig_t cfg = {};
-    cfg.gridDim = dim3(grid);
+    cfg.gridDim = dim3(grid * p.groups);
     cfg.blockDim = dim3(GEMM_THREADS);
     cfg.dynamicSmemBytes = smem;
     cfg.stream = s;

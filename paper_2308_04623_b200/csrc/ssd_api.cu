@@ -64,6 +64,7 @@ struct ssd_ctx {
     struct ForwardGraph { cudaGraph_t graph; cudaGraphExec_t exec; cudaGraphNode_t prep_node; int kernels; };
     ForwardGraph graphs[SSD_MAX_NODES + 1][3]; // (second index: the attention's key splits, 1 / 2 / 4 - chosen from the prefix length at each call)
     int attn_splits;                           // 0 = choose; 1, 2, 4 = always that many
+    int node_groups;                           // trees of more than 64 nodes: the layers' projections run on node groups of 64
     cudaStream_t capture_stream;
     AcceptScratch acc;
     int32_t *h_result; // pinned host copy of acc.result
@@ -340,18 +341,25 @@ cudaError_t enqueue_forward(ssd_ctx *ctx, int n, int cap, const NodeList &tk, co
             ctx->trace_count = ctx->trace_kernels ? 8 * *kernels : 0;
             return cudaSuccess;
         }
+        // Trees of more than 128 nodes: the layers' projections work on node groups of 64 (the grid is one 64-node arrangement per
+        // group, two CTAs per SM), with activation boxes of 64 rows.  Measured at the GPT-2-large shape (verify, us, without / with):
+        // 96 nodes 1565 / 1562, 128 nodes 1903 / 1917, 192 nodes 2563 / 2206, 256 nodes 3180 / 2640.
+        const int gr = (ctx->node_groups && n > 128) ? 64 : 0;
+        const ssd_ctx::ActMaps *ag = gr ? act_maps_pad(ctx, gr) : am;
+        if (!ag) return cudaErrorUnknown;
+        const int lgrid = gr ? (ctx->gemm_grid > 0 ? ctx->gemm_grid : 2 * sms) : grid;
         for (int l = 0; l < c.n_layer; ++l) {
             const LayerWeights &L = ctx->layers[l];
             const TensorMap *t = &ctx->map_layers[(size_t)4 * l];
             Q(launch_ln_prep(ctx->x, L.ln1_g, L.ln1_b, n, d, c.ln_eps, ctx->a_hi, a_lo, ctx->qkv, 3 * d, info, 0, pdl, s, trace_slot(ctx, *kernels)));
-            Q(launch_gemm_ws(&t[0], &am->a_hi, &am->a_pair, ctx->qkv, info, 3 * d, L.b_qkv, n, d, 3 * d, lo, grid, sms, ctx->d_status, pdl, s, trace_slot(ctx, *kernels)));
+            Q(launch_gemm_ws(&t[0], &ag->a_hi, &ag->a_pair, ctx->qkv, info, 3 * d, L.b_qkv, n, d, 3 * d, lo, lgrid, sms, ctx->d_status, pdl, s, trace_slot(ctx, *kernels), nullptr, nullptr, 0, 4, gr));
             if (staged) Q(launch_kv_stage(ctx->qkv, info, l * layer_elems, n, c.n_head, cap, pdl, s, trace_slot(ctx, *kernels)));
             Q(launch_tree_attention_mma(ctx->qkv, info, l * layer_elems, ctx->meta, n, c.n_head, cap, ctx->o_hi, o_lo, pdl, s, trace_slot(ctx, *kernels), ctx->attn_lo != 0, nullptr, 0, staged, attn_splits));
-            Q(launch_gemm_ws(&t[1], &am->o_hi, &am->o_pair, ctx->x, info, d, L.b_o, n, d, d, lo, grid, sms, ctx->d_status, pdl, s, trace_slot(ctx, *kernels)));
+            Q(launch_gemm_ws(&t[1], &ag->o_hi, &ag->o_pair, ctx->x, info, d, L.b_o, n, d, d, lo, lgrid, sms, ctx->d_status, pdl, s, trace_slot(ctx, *kernels), nullptr, nullptr, 0, 4, gr));
             Q(launch_ln_prep(ctx->x, L.ln2_g, L.ln2_b, n, d, c.ln_eps, ctx->a_hi, a_lo, ctx->h, F, info, 0, pdl, s, trace_slot(ctx, *kernels)));
-            Q(launch_gemm_ws(&t[2], &am->a_hi, &am->a_pair, ctx->h, info, F, L.b_fc, n, d, F, lo, grid, sms, ctx->d_status, pdl, s, trace_slot(ctx, *kernels)));
+            Q(launch_gemm_ws(&t[2], &ag->a_hi, &ag->a_pair, ctx->h, info, F, L.b_fc, n, d, F, lo, lgrid, sms, ctx->d_status, pdl, s, trace_slot(ctx, *kernels), nullptr, nullptr, 0, 4, gr));
             Q(launch_gelu_prep(ctx->h, n, F, ctx->h_hi, h_lo, pdl, s, trace_slot(ctx, *kernels)));
-            Q(launch_gemm_ws(&t[3], &am->h_hi, &am->h_pair, ctx->x, info, d, L.b_proj, n, F, d, lo, grid, sms, ctx->d_status, pdl, s, trace_slot(ctx, *kernels)));
+            Q(launch_gemm_ws(&t[3], &ag->h_hi, &ag->h_pair, ctx->x, info, d, L.b_proj, n, F, d, lo, lgrid, sms, ctx->d_status, pdl, s, trace_slot(ctx, *kernels), nullptr, nullptr, 0, 4, gr));
         }
         Q(launch_ln_prep(ctx->x, ctx->lnf_g, ctx->lnf_b, n, d, c.ln_eps, ctx->a_hi, a_lo, nullptr, 0, info, 0, pdl, s, trace_slot(ctx, *kernels)));
         Q(launch_gemm_ws(&ctx->map_wte, &am->a_hi, &am->a_pair, nullptr, info, c.vocab, nullptr, n, d, c.vocab, lo, hgrid, sms, ctx->d_status, pdl, s, trace_slot(ctx, *kernels), head));
@@ -474,6 +482,7 @@ int ssd_create(const ssd_config *cfg, int device, void *cuda_stream, ssd_ctx **o
     ctx->wte8 = nullptr; ctx->wte_scale = nullptr;
     ctx->w8_planes = 4;
     ctx->attn_splits = 0;
+    ctx->node_groups = 1;
     ctx->stage_kv_from = 128; // (measured at the GPT-2-large shape: 2 % faster at 128 nodes, 14 % at 256, slower below)
     ctx->device = device;
     ctx->stream = (cudaStream_t)cuda_stream;
@@ -1006,6 +1015,7 @@ int ssd_set_tuning(ssd_ctx *ctx, int32_t knob, int32_t value) {
     case SSD_TUNE_ATTN_LOW_PLANE: if (value != 0 && value != 1) return SSD_ERR_BAD_ARG; ctx->attn_lo = value; break;
     case SSD_TUNE_HEAD_STATS: if (value != 0 && value != 1) return SSD_ERR_BAD_ARG; ctx->use_head_stats = value; ctx->head_logits = nullptr; break;
     case SSD_TUNE_STAGE_KV_FROM: if (value < 0 || value > SSD_MAX_NODES + 1) return SSD_ERR_BAD_ARG; ctx->stage_kv_from = value; break;
+    case SSD_TUNE_NODE_GROUPS: if (value != 0 && value != 1) return SSD_ERR_BAD_ARG; ctx->node_groups = value; break;
     case SSD_TUNE_ATTN_SPLITS: if (value != 0 && value != 1 && value != 2 && value != 4) return SSD_ERR_BAD_ARG; ctx->attn_splits = value; break;
     case SSD_TUNE_W8_PLANES:
         if (!ctx->w8 || value < 2 || value > 4) return SSD_ERR_BAD_ARG;

@@ -95,11 +95,13 @@ cudaError_t prep_kernels_prepare();
 // activations e4m3 planes, the first w8_planes of the four (map_hi from make_tensor_map_u8_planes with that many planes per box;
 // map_lo unused); n <= 128 rows per launch, the rows
 // row0 .. row0 + n - 1 of the planes and of y; K need not be a multiple of 128; `head` is not supported.
+// With group_rows > 0 (a multiple of 16) and less than n, the nodes are cut into groups of that many and the grid is one copy of
+// the CTA arrangement per group (`grid` is the whole launch's CTA count); the maps' boxes then hold group_rows rows.  bf16 only.
 struct GemmHeadStats { float *val; int32_t *arg, *bad; };
 cudaError_t launch_gemm_ws(const void *map_w, const void *map_hi, const void *map_lo, float *y, const StepInfo *info, int ldy,
                            const float *bias, int n, int K, int out, int use_lo, int grid, int sm_count, int32_t *status, bool pdl,
                            cudaStream_t s, unsigned long long *trace = nullptr, const GemmHeadStats *head = nullptr,
-                           const float *w_scale = nullptr, int row0 = 0, int w8_planes = 4);
+                           const float *w_scale = nullptr, int row0 = 0, int w8_planes = 4, int group_rows = 0);
 // ---- projection with the split-K sums reduced inside a thread-block cluster (trees of up to 64 nodes) ----
 // What the epilogue does with the finished sums acc[i, o] (see k_gemm_cl.cu):
 enum { MODE_FOLD_STORE = 0, MODE_FOLD_GELU = 1, MODE_RESIDUAL = 2 };

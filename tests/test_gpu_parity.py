@@ -903,3 +903,27 @@ def test_attention_key_splits_merged_in_a_cluster(ssd, util, splits):
     assert np.abs(got - want).max() <= TOL_BF16
     assert p.ctx.device_status() == 0
     p.close()
+
+
+def test_projections_on_node_groups_give_the_same_logits(ssd, util):
+    """Trees of more than 128 nodes: the layers' projections run as one copy of a 64-node CTA arrangement per group of 64 nodes
+    (ragged last group included).  Against the oracle and against the whole-batch projections, with a commit in between."""
+    rng = np.random.default_rng(83)
+    p = util.Pair("ragged_bf16", seed=7, qk_gain=3.0)
+    V = p.V
+    p.prefill(ssd_synth.uniform_tokens(19, V, rng))
+    for n in (129, 200, 256, 193):
+        par = ssd_synth.tree_random(n, 7, rng)
+        tok = ssd_synth.uniform_tokens(n, V, rng)
+        p.ctx.set_tuning(ssd.SSD_TUNE_NODE_GROUPS, 1)
+        got, want, _ = p.verify(tok, par)
+        p.ctx.set_tuning(ssd.SSD_TUNE_NODE_GROUPS, 0)
+        plain, _, _ = p.verify(tok, par)
+        assert np.isfinite(got).all()
+        assert np.abs(got - want).max() <= TOL_BF16, n
+        assert np.abs(got - plain).max() <= 2e-3, n
+        p.ctx.set_tuning(ssd.SSD_TUNE_NODE_GROUPS, 1)
+        p.verify(tok, par)
+        p.commit(ssd_synth.path_to(par, n - 1))
+    assert p.ctx.device_status() == 0
+    p.close()
