@@ -348,6 +348,11 @@ cudaError_t enqueue_forward(ssd_ctx *ctx, int n, int cap, const NodeList &tk, co
         const ssd_ctx::ActMaps *ag = gr ? act_maps_pad(ctx, gr) : am;
         if (!ag) return cudaErrorUnknown;
         const int lgrid = gr ? (ctx->gemm_grid > 0 ? ctx->gemm_grid : 2 * sms) : grid;
+        // (the widest projection has so many output tiles that, times the groups of 64, every CTA would be left a tile's whole K -
+        //  a long chain of dependent units: it takes groups of 128 instead; measured 2640 -> 2548 us per verify at 256 nodes)
+        const int gr_fc = (gr && ((F + 127) / 128) * ((n + 63) / 64) > sms) ? 128 : gr;
+        const ssd_ctx::ActMaps *af = gr_fc == gr ? ag : act_maps_pad(ctx, gr_fc);
+        if (!af) return cudaErrorUnknown;
         for (int l = 0; l < c.n_layer; ++l) {
             const LayerWeights &L = ctx->layers[l];
             const TensorMap *t = &ctx->map_layers[(size_t)4 * l];
@@ -357,7 +362,7 @@ cudaError_t enqueue_forward(ssd_ctx *ctx, int n, int cap, const NodeList &tk, co
             Q(launch_tree_attention_mma(ctx->qkv, info, l * layer_elems, ctx->meta, n, c.n_head, cap, ctx->o_hi, o_lo, pdl, s, trace_slot(ctx, *kernels), ctx->attn_lo != 0, nullptr, 0, staged, attn_splits));
             Q(launch_gemm_ws(&t[1], &ag->o_hi, &ag->o_pair, ctx->x, info, d, L.b_o, n, d, d, lo, lgrid, sms, ctx->d_status, pdl, s, trace_slot(ctx, *kernels), nullptr, nullptr, 0, 4, gr));
             Q(launch_ln_prep(ctx->x, L.ln2_g, L.ln2_b, n, d, c.ln_eps, ctx->a_hi, a_lo, ctx->h, F, info, 0, pdl, s, trace_slot(ctx, *kernels)));
-            Q(launch_gemm_ws(&t[2], &ag->a_hi, &ag->a_pair, ctx->h, info, F, L.b_fc, n, d, F, lo, lgrid, sms, ctx->d_status, pdl, s, trace_slot(ctx, *kernels), nullptr, nullptr, 0, 4, gr));
+            Q(launch_gemm_ws(&t[2], &af->a_hi, &af->a_pair, ctx->h, info, F, L.b_fc, n, d, F, lo, lgrid, sms, ctx->d_status, pdl, s, trace_slot(ctx, *kernels), nullptr, nullptr, 0, 4, gr_fc));
             Q(launch_gelu_prep(ctx->h, n, F, ctx->h_hi, h_lo, pdl, s, trace_slot(ctx, *kernels)));
             Q(launch_gemm_ws(&t[3], &ag->h_hi, &ag->h_pair, ctx->x, info, d, L.b_proj, n, F, d, lo, lgrid, sms, ctx->d_status, pdl, s, trace_slot(ctx, *kernels), nullptr, nullptr, 0, 4, gr));
         }
