@@ -66,8 +66,7 @@ typedef struct {
  * without loss.  That instruction kind wants its other operand in an 8-bit format too, so the kernels that produce the
  * projections' inputs write each value as four e4m3 planes, x = 16 p0 + p1 + p2 / 16 + p3 / 256 to about 16
  * significant bits (what the bf16 model's hi + lo operand pair carries; |x| up to 7168 before the first plane
- * saturates); SSD_TUNE_W8_PLANES can drop the last ones.  A projection launch takes at most 128 nodes, so a larger
- * tree runs each projection as two launches.  The embedding look-up keeps the bf16 table; biases, LayerNorm
+ * saturates); SSD_TUNE_W8_PLANES can drop the last ones.  The embedding look-up keeps the bf16 table; biases, LayerNorm
  * parameters, the attention and the cache are as with dtype 1.  SSD_TUNE_CLUSTER_REDUCE and SSD_TUNE_HEAD_STATS
  * have no effect on such a context.
  */

@@ -34,7 +34,7 @@
 //     about 16 significant bits, what the bf16 hi + lo pair carries); the planes are stacked along N, so one
 //     instruction multiplies a weight slice by all four (N = 4 n_pad <= 256; two instructions for 128 rows), each
 //     plane's product in accumulator columns of its own.  The epilogue adds the four with their powers of two and
-//     multiplies by the row's scale.  At most 128 rows per launch (512 accumulator columns).
+//     multiplies by the row's scale.  At most 128 rows per node group (512 accumulator columns).
 //   * large trees: the nodes are cut into GROUPS of 64 and the grid is `groups` copies of the CTA arrangement of a
 //     64-node tree, copy g working on nodes 64 g .. 64 g + 63 (its activation boxes start at that row, its sums go
 //     to those rows of Y).  The weights are not read more often for it - the copies run at the same time and the
@@ -488,10 +488,10 @@ cudaError_t launch_gemm_ws(const void *map_w, const void *map_hi, const void *ma
                            const float *bias, int n, int K, int out, int use_lo, int grid, int sm_count, int32_t *status, bool pdl,
                            cudaStream_t s, unsigned long long *trace, const GemmHeadStats *head, const float *w_scale, int row0, int w8_planes, int group_rows) {
     const bool w8 = w_scale != nullptr; // map_w: the codes; map_hi: the four activation planes
-    if (w8 && (n > 128 || head || w8_planes < 2 || w8_planes > W8_PLANES)) return cudaErrorInvalidValue;
     // node groups: the activation maps' boxes hold group_rows rows (a multiple of 16), fewer than the tree has nodes
     const bool grouped = group_rows > 0 && group_rows < n;
-    if (grouped && (w8 || head || (group_rows & 15) || row0 != 0)) return cudaErrorInvalidValue;
+    if (grouped && (head || (group_rows & 15) || row0 != 0)) return cudaErrorInvalidValue;
+    if (w8 && ((grouped ? group_rows : n) > 128 || head || w8_planes < 2 || w8_planes > W8_PLANES)) return cudaErrorInvalidValue;
     GemmParams p;
     p.trace = trace;
     p.y = y; p.info = info; p.bias = bias; p.n = n; p.n_pad = grouped ? group_rows : (n + 15) & ~15;

@@ -308,33 +308,30 @@ cudaError_t enqueue_forward(ssd_ctx *ctx, int n, int cap, const NodeList &tk, co
         const bool staged = ctx->stage_kv_from > 0 && n >= ctx->stage_kv_from;
         if (ctx->w8) {
             // 8-bit weights: the same eight launches per layer; the element-wise kernels and the attention write four e4m3 planes,
-            // the projections run on the 8-bit tensor-core kind.  A projection takes at most 128 nodes (512 accumulator columns):
-            // a larger tree runs each projection as two launches over the two halves of the nodes.
+            // the projections run on the 8-bit tensor-core kind.  A CTA takes at most 128 nodes (512 accumulator columns); trees of
+            // more than 64 nodes run on node groups of 64 (256 columns: two CTAs per SM), like the bf16 model's large trees.
             const size_t rows = ctx->plane_rows, sa = rows * (size_t)d, sh = rows * (size_t)F;
-            const int n1 = n > 128 ? 128 : n, n2 = n - n1;
-            const ssd_ctx::ActMaps *m1 = act_maps_for(ctx, n1), *m2 = n2 ? act_maps_for(ctx, n2) : nullptr;
-            if (!m1 || (n2 && !m2)) return cudaErrorUnknown;
+            const int g8 = n > 64 ? 64 : 0;
+            const ssd_ctx::ActMaps *m1 = g8 ? act_maps_pad(ctx, g8) : am;
+            if (!m1) return cudaErrorUnknown;
+            const int grid8 = g8 ? (ctx->gemm_grid > 0 ? ctx->gemm_grid : 2 * sms) : grid;
             auto gemm8 = [&](const TensorMap *w, const TensorMap ssd_ctx::ActMaps::*act, float *y, int ldy, const float *bias, int K, int out, int g,
                              const float *scale) -> cudaError_t {
-                cudaError_t e8 = launch_gemm_ws(w, &(m1->*act), nullptr, y, info, ldy, bias, n1, K, out, 0, g, sms, ctx->d_status, pdl, s, trace_slot(ctx, *kernels), nullptr, scale, 0, ctx->w8_planes);
-                if (e8 == cudaSuccess && n2) {
-                    ++*kernels;
-                    e8 = launch_gemm_ws(w, &(m2->*act), nullptr, y, info, ldy, bias, n2, K, out, 0, g, sms, ctx->d_status, pdl, s, trace_slot(ctx, *kernels), nullptr, scale, n1, ctx->w8_planes);
-                }
-                return e8;
+                return launch_gemm_ws(w, &(m1->*act), nullptr, y, info, ldy, bias, n, K, out, 0, g, sms, ctx->d_status, pdl, s, trace_slot(ctx, *kernels), nullptr, scale, 0,
+                                      ctx->w8_planes, g8);
             };
             for (int l = 0; l < c.n_layer; ++l) {
                 const LayerWeights &L = ctx->layers[l];
                 const TensorMap *t = &ctx->map_layers[(size_t)4 * l];
                 Q(launch_ln_prep(ctx->x, L.ln1_g, L.ln1_b, n, d, c.ln_eps, nullptr, nullptr, ctx->qkv, 3 * d, info, 0, pdl, s, trace_slot(ctx, *kernels), ctx->a8, sa));
-                Q(gemm8(&t[0], &ssd_ctx::ActMaps::a_hi, ctx->qkv, 3 * d, L.b_qkv, d, 3 * d, grid, L.s_qkv));
+                Q(gemm8(&t[0], &ssd_ctx::ActMaps::a_hi, ctx->qkv, 3 * d, L.b_qkv, d, 3 * d, grid8, L.s_qkv));
                 if (staged) Q(launch_kv_stage(ctx->qkv, info, l * layer_elems, n, c.n_head, cap, pdl, s, trace_slot(ctx, *kernels)));
                 Q(launch_tree_attention_mma(ctx->qkv, info, l * layer_elems, ctx->meta, n, c.n_head, cap, nullptr, nullptr, pdl, s, trace_slot(ctx, *kernels), ctx->attn_lo != 0, ctx->o8, sa, staged, attn_splits));
-                Q(gemm8(&t[1], &ssd_ctx::ActMaps::o_hi, ctx->x, d, L.b_o, d, d, grid, L.s_o));
+                Q(gemm8(&t[1], &ssd_ctx::ActMaps::o_hi, ctx->x, d, L.b_o, d, d, grid8, L.s_o));
                 Q(launch_ln_prep(ctx->x, L.ln2_g, L.ln2_b, n, d, c.ln_eps, nullptr, nullptr, ctx->h, F, info, 0, pdl, s, trace_slot(ctx, *kernels), ctx->a8, sa));
-                Q(gemm8(&t[2], &ssd_ctx::ActMaps::a_hi, ctx->h, F, L.b_fc, d, F, grid, L.s_fc));
+                Q(gemm8(&t[2], &ssd_ctx::ActMaps::a_hi, ctx->h, F, L.b_fc, d, F, grid8, L.s_fc));
                 Q(launch_gelu_prep(ctx->h, n, F, nullptr, nullptr, pdl, s, trace_slot(ctx, *kernels), ctx->h8, sh));
-                Q(gemm8(&t[3], &ssd_ctx::ActMaps::h_hi, ctx->x, d, L.b_proj, F, d, grid, L.s_proj));
+                Q(gemm8(&t[3], &ssd_ctx::ActMaps::h_hi, ctx->x, d, L.b_proj, F, d, grid8, L.s_proj));
             }
             Q(launch_ln_prep(ctx->x, ctx->lnf_g, ctx->lnf_b, n, d, c.ln_eps, nullptr, nullptr, nullptr, 0, info, 0, pdl, s, trace_slot(ctx, *kernels), ctx->a8, sa));
             Q(gemm8(&ctx->map_wte, &ssd_ctx::ActMaps::a_hi, nullptr, c.vocab, nullptr, d, c.vocab, hgrid, ctx->wte_scale));

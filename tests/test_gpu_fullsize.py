@@ -103,7 +103,7 @@ def test_gpt2_xl_shape_random_trees():
 
 def test_gpt2_large_shape_8bit_weights():
     """The benchmark's shape with the streamed matrices as 8-bit codes (model on the code grid, so that the oracle holds the same
-    numbers): the 32-node tree bench.py times and a 160-node tree, which runs every projection as two launches."""
+    numbers): the 32-node tree bench.py times and a 160-node tree, whose projections run on node groups of 64."""
     def trees(p, rng):
         yield "n=32", ssd_synth.uniform_tokens(32, p.V, rng), ssd_synth.tree_branching(32, (4, 2, 2, 1, 1))
         yield "n=160", ssd_synth.uniform_tokens(160, p.V, rng), ssd_synth.tree_random(160, 8, rng)

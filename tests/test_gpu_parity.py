@@ -14,9 +14,8 @@ TOL_BF16 = 3e-2  # bf16 weights (stated target)
 
 def forward_launches(n_layer, n, w8=False):
     """Kernels of one default-path bf16 forward: tree preparation, clearing of the logits, embedding; eight per layer - nine from 128
-    nodes on, where a kernel of its own writes the tree's K / V rows to the cache; final LayerNorm and LM head.  With 8-bit weights a
-    projection takes 128 nodes per launch, so larger trees run each of the 4 L + 1 projections twice."""
-    return 3 + (8 + (1 if n >= 128 else 0)) * n_layer + 2 + ((4 * n_layer + 1) if (w8 and n > 128) else 0)
+    nodes on, where a kernel of its own writes the tree's K / V rows to the cache; final LayerNorm and LM head."""
+    return 3 + (8 + (1 if n >= 128 else 0)) * n_layer + 2
 
 
 @pytest.fixture(scope="module")
@@ -776,7 +775,6 @@ def test_w8_logits_against_the_oracle_and_the_bf16_path(ssd, util, cfg_name, qk_
         tok = ssd_synth.uniform_tokens(n, V, rng)
         before = p8.ctx.kernel_launches()
         got8, want, buf8 = p8.verify(tok, par)
-        # (a projection on the 8-bit tensor-core kind takes 128 nodes at most: larger trees run each one as two launches)
         assert p8.ctx.kernel_launches() - before == forward_launches(L, n, w8=True)
         got16, _, _ = p16.verify(tok, par)
         assert np.isfinite(got8).all()
