@@ -280,7 +280,7 @@ int ssd_kv_read(ssd_ctx *ctx, const ssd_kv *kv, int32_t layer, int32_t which, in
  *                                 (otherwise each 16-node tile of a head converts and stages the whole tree's keys itself); 0 = never
  *   SSD_TUNE_ATTN_SPLITS [0]      bf16 models: CTAs (one thread-block cluster) that share a (head, 16-node tile) of the attention, each
  *                                 with a part of the keys, merged in the first one's shared memory: 1, 2 or 4; 0 = from the prefix
- *                                 length of each call (1 up to 27 key blocks of 16, 2 up to 54, else 4)
+ *                                 length of each call (1 up to 19 key blocks of 16, 2 up to 27, else 4)
  *   SSD_TUNE_NODE_GROUPS [1]      bf16 models, trees of more than 128 nodes: the layers' projections run on node groups of 64 (one
  *                                 copy of a 64-node tree's CTA arrangement per group) instead of on the whole batch per CTA
  *   SSD_TUNE_KERNEL_TRACE [0]     record a timeline of every kernel of a bf16 forward (see ssd_get_phase_trace)

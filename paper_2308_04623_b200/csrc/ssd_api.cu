@@ -225,7 +225,7 @@ static int attn_splits_for(const ssd_ctx *ctx, int kv_len, int n) {
     int s = ctx->attn_splits;
     if (s == 0) {
         const int blocks = (kv_len + n + 15) / 16;
-        s = blocks > 54 ? 4 : blocks > 27 ? 2 : 1;
+        s = blocks > 27 ? 4 : blocks > 19 ? 2 : 1;
     }
     while (s > 1 && (staged || ctas * s > ctx->sm_count)) s >>= 1; // (an attention CTA has an SM to itself: more CTAs than SMs run in waves)
     return s;
