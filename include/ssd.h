@@ -283,11 +283,15 @@ int ssd_kv_read(ssd_ctx *ctx, const ssd_kv *kv, int32_t layer, int32_t which, in
  *                                 length of each call (1 up to 19 key blocks of 16, 2 up to 27, else 4)
  *   SSD_TUNE_NODE_GROUPS [1]      bf16 models, trees of more than 128 nodes: the layers' projections run on node groups of 64 (one
  *                                 copy of a 64-node tree's CTA arrangement per group) instead of on the whole batch per CTA
+ *   SSD_TUNE_FUSED_GELU [0]       bf16 models, both planes, at most 64 nodes per CTA of the projections: the feed-forward block's
+ *                                 back-projection reads the fp32 sums of the first projection and makes its gelu(.) operand planes
+ *                                 itself (one kernel fewer per layer; same values; measured slower: every output tile's CTAs
+ *                                 convert the same values again); 0 = a separate element-wise kernel writes them
  *   SSD_TUNE_KERNEL_TRACE [0]     record a timeline of every kernel of a bf16 forward (see ssd_get_phase_trace)
  */
 enum { SSD_TUNE_LOW_PLANE = 0, SSD_TUNE_DEPENDENT_LAUNCH = 1, SSD_TUNE_GRAPH = 2, SSD_TUNE_GEMM_CTAS = 3, SSD_TUNE_CLUSTER_REDUCE = 4,
        SSD_TUNE_CLUSTER_MAX = 5, SSD_TUNE_ATTN_LOW_PLANE = 6, SSD_TUNE_HEAD_CTAS = 7, SSD_TUNE_KERNEL_TRACE = 8, SSD_TUNE_CLUSTER_QKV = 9, SSD_TUNE_CLUSTER_O = 10,
-       SSD_TUNE_CLUSTER_FC = 11, SSD_TUNE_CLUSTER_PROJ = 12, SSD_TUNE_HEAD_STATS = 13, SSD_TUNE_W8_PLANES = 14, SSD_TUNE_STAGE_KV_FROM = 15, SSD_TUNE_ATTN_SPLITS = 16, SSD_TUNE_NODE_GROUPS = 17 };
+       SSD_TUNE_CLUSTER_FC = 11, SSD_TUNE_CLUSTER_PROJ = 12, SSD_TUNE_HEAD_STATS = 13, SSD_TUNE_W8_PLANES = 14, SSD_TUNE_STAGE_KV_FROM = 15, SSD_TUNE_ATTN_SPLITS = 16, SSD_TUNE_NODE_GROUPS = 17, SSD_TUNE_FUSED_GELU = 18 };
 int ssd_set_tuning(ssd_ctx *ctx, int32_t knob, int32_t value);
 
 /*

@@ -46,6 +46,7 @@
 
 #include "sm100_ptx.cuh"
 #include "ssd_internal.h"
+#include "act_math.cuh"
 
 namespace {
 constexpr int TILE_M = 128;                 // output features per tile (MMA M)
@@ -93,6 +94,7 @@ struct __align__(8) Barriers {
     uint64_t empty[MAX_STAGES];
     uint64_t acc_full[2];
     uint64_t acc_empty[2];
+    uint64_t b_full[MAX_STAGES];        // ACT: the epilogue warps have written a stage's activation planes
     uint32_t tmem_base;
     uint32_t abort;
 };
@@ -106,7 +108,12 @@ __device__ __forceinline__ void fail(const GemmParams &p, Barriers *b, int code)
 
 
 // (Few enough registers for three CTAs of it, or two next to the element-wise kernels' CTAs, to be resident on an SM.)
-template <bool W8>
+// ACT (bf16 weights, hi + lo planes, tile-aligned split, at most 64 rows per node group): the activations are not read as
+// prepared planes; `map_hi` is the fp32 matrix the previous projection accumulated into, its [n_pad x 64] block of a stage
+// lands where the two planes will be (the same bytes), and the epilogue warps - idle until the accumulator completes - turn
+// it into gelu(.) as hi / lo planes in the swizzled layout the MMA reads.  That removes a kernel, and with it one
+// hand-over between dependent kernels per layer, from the chain.
+template <bool W8, bool ACT>
 __global__ void __launch_bounds__(GEMM_THREADS, 3)
 gemm_ws_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant__ CUtensorMap map_hi,
                const __grid_constant__ CUtensorMap map_lo, const GemmParams p) {
@@ -150,6 +157,7 @@ gemm_ws_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant_
         ptx::trace_mark(p.trace, 0);
         for (int s = 0; s < p.stages; ++s) { ptx::mbar_init(&bars->full[s], 1); ptx::mbar_init(&bars->empty[s], 1); }
         for (int a = 0; a < 2; ++a) { ptx::mbar_init(&bars->acc_full[a], 1); ptx::mbar_init(&bars->acc_empty[a], 4); }
+        if (ACT) for (int s = 0; s < p.stages; ++s) ptx::mbar_init(&bars->b_full[s], 4);
         // a device error recorded by an earlier kernel makes every later one a no-op, so that a
         // failure costs one time-out, not one per launch
         bars->abort = (*reinterpret_cast<volatile int32_t *>(p.status) != 0) ? 1u : 0u;
@@ -185,7 +193,7 @@ gemm_ws_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant_
     } else if (warp == 0) {
         // ===================== TMA producer =====================
         if (lane == 0 && u1 > u0) {
-            if (W8 || !p.use_lo) ptx::prefetch_tensormap(&map_hi);
+            if (W8 || ACT || !p.use_lo) ptx::prefetch_tensormap(&map_hi);
             else ptx::prefetch_tensormap(&map_lo);
             const uint64_t pol = ptx::policy_evict_first();
             const uint32_t tx = (uint32_t)stage_bytes;
@@ -208,6 +216,8 @@ gemm_ws_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant_
                 // (the activation maps' box is the whole padded batch: one operation per plane; W8: one for the four planes)
                 if (W8) {
                     ptx::tma_load_3d(st + A_BYTES, &map_hi, kt * KT, row0, 0, &bars->full[s]);
+                } else if (ACT) { // the fp32 block [n_pad x 64]: as many bytes as the two planes made from it
+                    ptx::tma_load_2d(st + A_BYTES, &map_hi, kt * TILE_K, row0, &bars->full[s]);
                 } else {
                     // (with the lo plane: ONE box over both planes - they are adjacent in memory as in the stage - since every copy
                     //  this one thread issues costs it some 50-100 ns ahead of the first MMA)
@@ -242,6 +252,7 @@ gemm_ws_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant_
                     ptx::tc_fence_after_sync();
                 }
                 if (!ptx::mbar_wait_bounded(&bars->full[s], round & 1)) { fail(p, bars, 0x300 + s); ok = false; break; }
+                if (ACT && !ptx::mbar_wait_bounded(&bars->b_full[s], round & 1)) { fail(p, bars, 0x500 + s); ok = false; break; }
                 // (no tcgen05 fence here: the stage was filled through the asynchronous proxy and its completion observed on
                 //  the mbarrier; a fence per unit made the issuing thread wait out the MMAs in flight, ~0.6 us each time)
                 const uint32_t a_addr = ptx::smem_u32(smem + (size_t)s * stage_bytes);
@@ -273,6 +284,49 @@ gemm_ws_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant_
         const int et = threadIdx.x - 64; // 0..127 among the epilogue threads
         int seg = 0;
         bool ok = true;
+        if (ACT) {
+            // Stage by stage: wait for the fp32 block, take it into registers (thread -> (row, 8 columns): 32 bytes), meet - the
+            // planes overwrite the block - then write gelu(.) as bf16 hi and lo, 16 bytes each, where the 128-byte swizzle puts
+            // chunk c of row r: at chunk c ^ (r & 7).  Rows past the tree (or the group) become zeros.
+            const int iters = p.n_pad >> 4;     // 8 chunks per row, 128 threads: n_pad / 16 chunks per thread (at most 4)
+            int s = 0, round = 0;
+            for (int u = u0; u < u1; ++u) {
+                int good = 1;
+                if (lane == 0) good = ptx::mbar_wait_bounded<EPI_POLL_NS>(&bars->full[s], round & 1) ? 1 : 0;
+                good = __shfl_sync(0xffffffffu, good, 0);
+                if (!good && lane == 0) fail(p, bars, 0x600 + s);
+                uint8_t *const blk = smem + (size_t)s * stage_bytes + A_BYTES;
+                float4 v[4][2];
+#pragma unroll
+                for (int it = 0; it < 4; ++it)
+                    if (it < iters && good) {
+                        const int id = et + it * 128, r = id >> 3, c = id & 7;
+                        const float4 *src = reinterpret_cast<const float4 *>(blk + r * 256 + c * 32);
+                        v[it][0] = src[0]; v[it][1] = src[1];
+                    }
+                epi_sync();
+                if (*reinterpret_cast<volatile uint32_t *>(&bars->abort)) { ok = false; break; } // (the same answer in all four warps)
+#pragma unroll
+                for (int it = 0; it < 4; ++it)
+                    if (it < iters) {
+                        const int id = et + it * 128, r = id >> 3, c = id & 7;
+                        uint4 hi = make_uint4(0u, 0u, 0u, 0u), lo = hi;
+                        if (r < n_rows) {
+                            const float g[8] = {act::gelu_tanh_fast(v[it][0].x), act::gelu_tanh_fast(v[it][0].y), act::gelu_tanh_fast(v[it][0].z),
+                                                act::gelu_tanh_fast(v[it][0].w), act::gelu_tanh_fast(v[it][1].x), act::gelu_tanh_fast(v[it][1].y),
+                                                act::gelu_tanh_fast(v[it][1].z), act::gelu_tanh_fast(v[it][1].w)};
+                            act::split8_bf16(g, hi, lo);
+                        }
+                        const int at = r * 128 + ((c ^ (r & 7)) << 4);
+                        *reinterpret_cast<uint4 *>(blk + at) = hi;
+                        *reinterpret_cast<uint4 *>(blk + b_bytes + at) = lo;
+                    }
+                ptx::fence_proxy_async_smem(); // the tensor cores read shared memory through the asynchronous proxy
+                __syncwarp();
+                if (lane == 0) ptx::mbar_arrive(&bars->b_full[s]);
+                if (++s == p.stages) { s = 0; ++round; }
+            }
+        }
         for (int u = u0; u < u1;) { // (no early exit: the four warps must meet at the same barriers)
             const int tile = u / p.k_tiles;
             const int seg_end = min(u1, (tile + 1) * p.k_tiles);
@@ -477,16 +531,33 @@ int gemm_ws_stages(int n_pad, int planes, bool shared_sm) {
 }
 
 cudaError_t gemm_ws_prepare() {
-    cudaError_t e = cudaFuncSetAttribute(gemm_ws_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024);
-    if (e == cudaSuccess) e = cudaFuncSetAttribute(gemm_ws_kernel<false>, cudaFuncAttributePreferredSharedMemoryCarveout, cudaSharedmemCarveoutMaxShared);
-    if (e == cudaSuccess) e = cudaFuncSetAttribute(gemm_ws_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024);
-    if (e == cudaSuccess) e = cudaFuncSetAttribute(gemm_ws_kernel<true>, cudaFuncAttributePreferredSharedMemoryCarveout, cudaSharedmemCarveoutMaxShared);
+    cudaError_t e = cudaSuccess;
+    const void *kernels[] = {(const void *)gemm_ws_kernel<false, false>, (const void *)gemm_ws_kernel<true, false>, (const void *)gemm_ws_kernel<false, true>};
+    for (const void *k : kernels) {
+        if (e == cudaSuccess) e = cudaFuncSetAttribute(k, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024);
+        if (e == cudaSuccess) e = cudaFuncSetAttribute(k, cudaFuncAttributePreferredSharedMemoryCarveout, cudaSharedmemCarveoutMaxShared);
+    }
     return e;
+}
+
+// An fp32 row-major matrix [rows, cols] (cols a multiple of 64) as a 2-D tensor map with boxes of [box_rows, 64], not
+// swizzled; out-of-range rows read as zero.
+int make_tensor_map_f32(void *map_out, const void *base, uint64_t rows, uint64_t cols, uint32_t box_rows) {
+    EncodeTiledFn fn = encode_fn();
+    if (!fn) return SSD_ERR_CUDA;
+    cuuint64_t dims[2] = {cols, rows};
+    cuuint64_t strides[1] = {cols * 4};
+    cuuint32_t box[2] = {TILE_K, box_rows};
+    cuuint32_t estr[2] = {1, 1};
+    CUresult r = fn((CUtensorMap *)map_out, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 2, const_cast<void *>(base), dims, strides, box, estr,
+                    CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                    CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    return r == CUDA_SUCCESS ? SSD_OK : SSD_ERR_CUDA;
 }
 
 cudaError_t launch_gemm_ws(const void *map_w, const void *map_hi, const void *map_lo, float *y, const StepInfo *info, int ldy,
                            const float *bias, int n, int K, int out, int use_lo, int grid, int sm_count, int32_t *status, bool pdl,
-                           cudaStream_t s, unsigned long long *trace, const GemmHeadStats *head, const float *w_scale, int row0, int w8_planes, int group_rows) {
+                           cudaStream_t s, unsigned long long *trace, const GemmHeadStats *head, const float *w_scale, int row0, int w8_planes, int group_rows, int act_gelu) {
     const bool w8 = w_scale != nullptr; // map_w: the codes; map_hi: the four activation planes
     // node groups: the activation maps' boxes hold group_rows rows (a multiple of 16), fewer than the tree has nodes
     const bool grouped = group_rows > 0 && group_rows < n;
@@ -538,6 +609,8 @@ cudaError_t launch_gemm_ws(const void *map_w, const void *map_hi, const void *ma
     attr[0].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attr;
     cfg.numAttrs = pdl ? 1 : 0;
-    return cudaLaunchKernelEx(&cfg, w8 ? gemm_ws_kernel<true> : gemm_ws_kernel<false>, *(const CUtensorMap *)map_w,
+    // (fp32 source of the activations: one tile per CTA, both planes, a block a thread can hold its share of)
+    if (act_gelu && (w8 || head || !use_lo || p.split == 0 || p.n_pad > 64)) return cudaErrorInvalidValue;
+    return cudaLaunchKernelEx(&cfg, w8 ? gemm_ws_kernel<true, false> : act_gelu ? gemm_ws_kernel<false, true> : gemm_ws_kernel<false, false>, *(const CUtensorMap *)map_w,
                               *(const CUtensorMap *)map_hi, *(const CUtensorMap *)(map_lo ? map_lo : map_hi), p);
 }

@@ -11,6 +11,7 @@
 #include "sm100_ptx.cuh"
 #include "ssd_internal.h"
 #include "w8_planes.cuh"
+#include "act_math.cuh"
 
 namespace {
 __device__ __forceinline__ float block_sum_256(float v, float *red) {
@@ -29,10 +30,8 @@ __device__ __forceinline__ float block_sum_256(float v, float *red) {
 // The row is read once, as 16-byte vectors held in registers (d a multiple of 4, at most 4 * PER4 * 256: PER4 = 2 serves d <= 2048, PER4 = 8 the rest up to 8192), so the
 // kernel is one L2 round trip plus two block reductions; the code is kept small on purpose (these kernels run once
 // per layer between other kernels, and what they mostly wait for is their own instructions).
-__device__ __forceinline__ uint2 pack4_bf16(float a, float b, float c, float d) {
-    const __nv_bfloat162 lo = __floats2bfloat162_rn(a, b), hi = __floats2bfloat162_rn(c, d);
-    return make_uint2(*reinterpret_cast<const uint32_t *>(&lo), *reinterpret_cast<const uint32_t *>(&hi));
-}
+using act::pack4_bf16;
+using act::gelu_tanh_fast;
 template <int PER4, bool P8>
 __global__ void __launch_bounds__(256) ln_prep_kernel(const float *__restrict__ x, const float *__restrict__ g, const float *__restrict__ b,
                                                       int d, float eps, __nv_bfloat16 *__restrict__ a_hi, __nv_bfloat16 *__restrict__ a_lo,
@@ -104,10 +103,6 @@ __global__ void __launch_bounds__(256) ln_prep_kernel(const float *__restrict__ 
 
 // h = gelu(acc) -> bf16 hi/lo planes (acc already holds the bias); eight consecutive values per thread (count is a
 // multiple of 8: the feed-forward width is a multiple of 64)
-__device__ __forceinline__ float gelu_tanh_fast(float z) { // 0.5 z (1 + tanh u) = z / (1 + exp(-2u))
-    const float u2 = 1.5957691216057308f * (z + 0.044715f * z * z * z);
-    return __fdividef(z, 1.0f + __expf(-u2));
-}
 template <bool P8>
 __global__ void __launch_bounds__(256) gelu_prep_kernel(const float *__restrict__ acc, size_t count, __nv_bfloat16 *__restrict__ h_hi,
                                                         __nv_bfloat16 *__restrict__ h_lo, unsigned long long *trace, uint8_t *__restrict__ planes8,

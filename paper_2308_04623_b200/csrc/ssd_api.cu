@@ -36,7 +36,7 @@ struct ssd_ctx {
     __nv_bfloat16 *a_hi, *a_lo, *o_hi, *o_lo, *h_hi, *h_lo;
     // activation planes as tensor maps whose box is the whole padded batch [n_pad rows x 64]: one TMA operation per
     // plane and k tile (index n_pad / 16 - 1; built on first use)
-    struct ActMaps { TensorMap a_hi, a_lo, o_hi, o_lo, h_hi, h_lo, a_pair, o_pair, h_pair; bool built; }; // (_pair: hi and lo planes as one box)
+    struct ActMaps { TensorMap a_hi, a_lo, o_hi, o_lo, h_hi, h_lo, a_pair, o_pair, h_pair, h_src; bool built; }; // (_pair: hi and lo planes as one box)
     ActMaps act_maps[SSD_MAX_NODES / 16];
     size_t plane_rows;
     TensorMap map_wte;
@@ -64,6 +64,7 @@ struct ssd_ctx {
     struct ForwardGraph { cudaGraph_t graph; cudaGraphExec_t exec; cudaGraphNode_t prep_node; int kernels; };
     ForwardGraph graphs[SSD_MAX_NODES + 1][3]; // (second index: the attention's key splits, 1 / 2 / 4 - chosen from the prefix length at each call)
     int attn_splits;                           // 0 = choose; 1, 2, 4 = always that many
+    int fused_gelu;                            // the back-projection makes its gelu(.) operand planes itself (no separate kernel)
     int node_groups;                           // trees of more than 64 nodes: the layers' projections run on node groups of 64
     cudaStream_t capture_stream;
     AcceptScratch acc;
@@ -190,6 +191,7 @@ static const ssd_ctx::ActMaps *act_maps_pad(ssd_ctx *ctx, int n_pad) {
         if (m == SSD_OK) m = make_tensor_map_bf16_pair(&am.a_pair, ctx->a_hi, rows, d, n_pad);
         if (m == SSD_OK) m = make_tensor_map_bf16_pair(&am.o_pair, ctx->o_hi, rows, d, n_pad);
         if (m == SSD_OK) m = make_tensor_map_bf16_pair(&am.h_pair, ctx->h_hi, rows, F, n_pad);
+        if (m == SSD_OK) m = make_tensor_map_f32(&am.h_src, ctx->h, ctx->cfg.max_nodes, F, n_pad); // (the feed-forward sums themselves)
         if (m != SSD_OK) return nullptr;
         am.built = true;
     }
@@ -350,6 +352,14 @@ cudaError_t enqueue_forward(ssd_ctx *ctx, int n, int cap, const NodeList &tk, co
         const int gr_fc = (gr && ((F + 127) / 128) * ((n + 63) / 64) > sms) ? 128 : gr;
         const ssd_ctx::ActMaps *af = gr_fc == gr ? ag : act_maps_pad(ctx, gr_fc);
         if (!af) return cudaErrorUnknown;
+        // Opt-in: the back-projection reads the feed-forward sums and applies the GELU itself (the ACT instantiation of the kernel),
+        // when it runs with both planes, on at most 64 rows per CTA and with at least one CTA per output tile.  Measured slower
+        // (GPT-2-large shape, 32 nodes: 1166 against 1075 us per verify; 64 nodes 1459 / 1339; 256 nodes 2877 / 2541): every CTA of
+        // the ten output tiles converts the same slice again - two special-function operations per value, 0.35-0.7 us per k tile on
+        // one warp per scheduler, 3.9 us from dependencies to accumulator against 1.9 - and with no kernel between the two
+        // feed-forward projections the second one's CTAs find room, and start their weight loads, only as the first one's leave.
+        const int rows_cta = gr ? gr : (n + 15) & ~15;
+        const bool fuse_gelu = ctx->fused_gelu && lo && rows_cta <= 64 && lgrid / (gr ? (n + gr - 1) / gr : 1) >= (d + 127) / 128;
         for (int l = 0; l < c.n_layer; ++l) {
             const LayerWeights &L = ctx->layers[l];
             const TensorMap *t = &ctx->map_layers[(size_t)4 * l];
@@ -360,8 +370,12 @@ cudaError_t enqueue_forward(ssd_ctx *ctx, int n, int cap, const NodeList &tk, co
             Q(launch_gemm_ws(&t[1], &ag->o_hi, &ag->o_pair, ctx->x, info, d, L.b_o, n, d, d, lo, lgrid, sms, ctx->d_status, pdl, s, trace_slot(ctx, *kernels), nullptr, nullptr, 0, 4, gr));
             Q(launch_ln_prep(ctx->x, L.ln2_g, L.ln2_b, n, d, c.ln_eps, ctx->a_hi, a_lo, ctx->h, F, info, 0, pdl, s, trace_slot(ctx, *kernels)));
             Q(launch_gemm_ws(&t[2], &af->a_hi, &af->a_pair, ctx->h, info, F, L.b_fc, n, d, F, lo, lgrid, sms, ctx->d_status, pdl, s, trace_slot(ctx, *kernels), nullptr, nullptr, 0, 4, gr_fc));
-            Q(launch_gelu_prep(ctx->h, n, F, ctx->h_hi, h_lo, pdl, s, trace_slot(ctx, *kernels)));
-            Q(launch_gemm_ws(&t[3], &ag->h_hi, &ag->h_pair, ctx->x, info, d, L.b_proj, n, F, d, lo, lgrid, sms, ctx->d_status, pdl, s, trace_slot(ctx, *kernels), nullptr, nullptr, 0, 4, gr));
+            if (fuse_gelu) {
+                Q(launch_gemm_ws(&t[3], &ag->h_src, nullptr, ctx->x, info, d, L.b_proj, n, F, d, lo, lgrid, sms, ctx->d_status, pdl, s, trace_slot(ctx, *kernels), nullptr, nullptr, 0, 4, gr, 1));
+            } else {
+                Q(launch_gelu_prep(ctx->h, n, F, ctx->h_hi, h_lo, pdl, s, trace_slot(ctx, *kernels)));
+                Q(launch_gemm_ws(&t[3], &ag->h_hi, &ag->h_pair, ctx->x, info, d, L.b_proj, n, F, d, lo, lgrid, sms, ctx->d_status, pdl, s, trace_slot(ctx, *kernels), nullptr, nullptr, 0, 4, gr));
+            }
         }
         Q(launch_ln_prep(ctx->x, ctx->lnf_g, ctx->lnf_b, n, d, c.ln_eps, ctx->a_hi, a_lo, nullptr, 0, info, 0, pdl, s, trace_slot(ctx, *kernels)));
         Q(launch_gemm_ws(&ctx->map_wte, &am->a_hi, &am->a_pair, nullptr, info, c.vocab, nullptr, n, d, c.vocab, lo, hgrid, sms, ctx->d_status, pdl, s, trace_slot(ctx, *kernels), head));
@@ -485,6 +499,7 @@ int ssd_create(const ssd_config *cfg, int device, void *cuda_stream, ssd_ctx **o
     ctx->w8_planes = 4;
     ctx->attn_splits = 0;
     ctx->node_groups = 1;
+    ctx->fused_gelu = 0;
     ctx->stage_kv_from = 128; // (measured at the GPT-2-large shape: 2 % faster at 128 nodes, 14 % at 256, slower below)
     ctx->device = device;
     ctx->stream = (cudaStream_t)cuda_stream;
@@ -1018,6 +1033,7 @@ int ssd_set_tuning(ssd_ctx *ctx, int32_t knob, int32_t value) {
     case SSD_TUNE_HEAD_STATS: if (value != 0 && value != 1) return SSD_ERR_BAD_ARG; ctx->use_head_stats = value; ctx->head_logits = nullptr; break;
     case SSD_TUNE_STAGE_KV_FROM: if (value < 0 || value > SSD_MAX_NODES + 1) return SSD_ERR_BAD_ARG; ctx->stage_kv_from = value; break;
     case SSD_TUNE_NODE_GROUPS: if (value != 0 && value != 1) return SSD_ERR_BAD_ARG; ctx->node_groups = value; break;
+    case SSD_TUNE_FUSED_GELU: if (value != 0 && value != 1) return SSD_ERR_BAD_ARG; ctx->fused_gelu = value; break;
     case SSD_TUNE_ATTN_SPLITS: if (value != 0 && value != 1 && value != 2 && value != 4) return SSD_ERR_BAD_ARG; ctx->attn_splits = value; break;
     case SSD_TUNE_W8_PLANES:
         if (!ctx->w8 || value < 2 || value > 4) return SSD_ERR_BAD_ARG;

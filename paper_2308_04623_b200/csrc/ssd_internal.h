@@ -78,6 +78,7 @@ struct alignas(64) TensorMap { unsigned char bytes[128]; };
 int make_tensor_map_bf16(void *map_out, const void *base, uint64_t rows, uint64_t cols, uint32_t box_rows);
 int make_tensor_map_bf16_pair(void *map_out, const void *base, uint64_t rows, uint64_t cols, uint32_t box_rows);
 int make_tensor_map_u8(void *map_out, const void *base, uint64_t rows, uint64_t cols, uint32_t box_rows);
+int make_tensor_map_f32(void *map_out, const void *base, uint64_t rows, uint64_t cols, uint32_t box_rows); // boxes of [box_rows, 64], not swizzled
 int make_tensor_map_u8_planes(void *map_out, const void *base, uint64_t rows, uint64_t cols, uint32_t box_rows, uint32_t box_planes);
 // 8-bit weights: W[rows, cols] bf16 -> e4m3 codes [rows, cols] and one power-of-two scale per row, the smallest that brings the
 // row's largest magnitude within the format's range (448); code = round-to-nearest-even(W / scale).  A row of zeros gets scale 1.
@@ -97,11 +98,14 @@ cudaError_t prep_kernels_prepare();
 // row0 .. row0 + n - 1 of the planes and of y; K need not be a multiple of 128; `head` is not supported.
 // With group_rows > 0 (a multiple of 16) and less than n, the nodes are cut into groups of that many and the grid is one copy of
 // the CTA arrangement per group (`grid` is the whole launch's CTA count); the maps' boxes then hold group_rows rows.  bf16 only.
+// With act_gelu the activations are X = gelu(S), S the fp32 matrix [rows, K] behind map_hi (make_tensor_map_f32; map_lo unused):
+// the kernel makes the hi / lo planes itself, with the arithmetic of launch_gelu_prep.  Needs use_lo, at most 64 rows (per
+// group) and at least as many CTAs as output tiles; bf16 weights only.
 struct GemmHeadStats { float *val; int32_t *arg, *bad; };
 cudaError_t launch_gemm_ws(const void *map_w, const void *map_hi, const void *map_lo, float *y, const StepInfo *info, int ldy,
                            const float *bias, int n, int K, int out, int use_lo, int grid, int sm_count, int32_t *status, bool pdl,
                            cudaStream_t s, unsigned long long *trace = nullptr, const GemmHeadStats *head = nullptr,
-                           const float *w_scale = nullptr, int row0 = 0, int w8_planes = 4, int group_rows = 0);
+                           const float *w_scale = nullptr, int row0 = 0, int w8_planes = 4, int group_rows = 0, int act_gelu = 0);
 // ---- projection with the split-K sums reduced inside a thread-block cluster (trees of up to 64 nodes) ----
 // What the epilogue does with the finished sums acc[i, o] (see k_gemm_cl.cu):
 enum { MODE_FOLD_STORE = 0, MODE_FOLD_GELU = 1, MODE_RESIDUAL = 2 };

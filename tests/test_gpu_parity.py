@@ -903,6 +903,40 @@ def test_attention_key_splits_merged_in_a_cluster(ssd, util, splits):
     p.close()
 
 
+def test_back_projection_applies_the_gelu_itself(ssd, util):
+    """SSD_TUNE_FUSED_GELU = 1: the feed-forward block's back-projection reads the first projection's fp32 sums and writes its
+    gelu(.) hi / lo operand planes into shared memory itself, against the default, a separate element-wise kernel (same arithmetic,
+    so the logits differ by the order of the fp32 reductions only), and against the oracle; one launch fewer per layer where it
+    applies (at most 64 rows per CTA: trees of up to 64 nodes, node groups beyond 128).  Tree sizes with one to four 16-row chunks
+    per thread, ragged ones, and node groups with a ragged last group."""
+    rng = np.random.default_rng(97)
+    p = util.Pair("ragged_bf16", seed=9, qk_gain=3.0)
+    V, L = p.V, p.cfg["n_layer"]
+    p.prefill(ssd_synth.uniform_tokens(23, V, rng))
+    for n in (1, 16, 17, 33, 48, 64, 100, 150, 256):
+        par = ssd_synth.tree_random(n, 5, rng)
+        tok = ssd_synth.uniform_tokens(n, V, rng)
+        p.ctx.set_tuning(ssd.SSD_TUNE_FUSED_GELU, 0)
+        before = p.ctx.kernel_launches()
+        plain, want, _ = p.verify(tok, par)
+        separate = p.ctx.kernel_launches() - before
+        p.ctx.set_tuning(ssd.SSD_TUNE_FUSED_GELU, 1)
+        before = p.ctx.kernel_launches()
+        got, _, _ = p.verify(tok, par)
+        assert separate == forward_launches(L, n) and p.ctx.kernel_launches() - before == separate - (0 if 64 < n <= 128 else L), n
+        assert np.isfinite(got).all()
+        assert np.abs(got - want).max() <= TOL_BF16, n
+        assert np.abs(got - plain).max() <= 1e-3, n
+        p.commit(ssd_synth.path_to(par, n - 1))
+    # without the low plane the projection keeps reading prepared planes
+    p.ctx.set_tuning(ssd.SSD_TUNE_LOW_PLANE, 0)
+    before = p.ctx.kernel_launches()
+    p.verify(tok[:20], ssd_synth.tree_random(20, 5, rng))
+    assert p.ctx.kernel_launches() - before == forward_launches(L, 20)
+    assert p.ctx.device_status() == 0
+    p.close()
+
+
 def test_projections_on_node_groups_give_the_same_logits(ssd, util):
     """Trees of more than 128 nodes: the layers' projections run as one copy of a 64-node CTA arrangement per group of 64 nodes
     (ragged last group included).  Against the oracle and against the whole-batch projections, with a commit in between."""
