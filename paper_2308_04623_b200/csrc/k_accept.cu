@@ -110,7 +110,8 @@ __global__ void greedy_walk_kernel(NodeList tokens, NodeList parent, int n, int 
 struct BlockScratch {
     double d[32];
     int i[32];
-    unsigned hist[256];
+    unsigned hist[2048];  // radix selection: counts per digit (up to 11 bits a round)
+    unsigned cand[4096];  // ... and the keys still in the running after the first round
     unsigned sel_prefix, sel_k;
     int flag;
 };
@@ -159,35 +160,129 @@ __device__ __forceinline__ float from_orderable(unsigned u) {
 }
 
 // k-th largest value of z[0..V) by most-significant-digit radix selection (exact, integer work).
-__device__ float kth_largest(const float *__restrict__ z, int V, int k, BlockScratch &s) {
-    if (threadIdx.x == 0) { s.sel_prefix = 0u; s.sel_k = (unsigned)k; }
-    for (int shift = 24; shift >= 0; shift -= 8) {
-        for (int b = threadIdx.x; b < 256; b += ACC_THREADS) s.hist[b] = 0u;
-        __syncthreads();
-        const unsigned prefix = s.sel_prefix;
-        const unsigned himask = (shift == 24) ? 0u : (0xffffffffu << (shift + 8));
-        // (logits share their leading bytes, so most keys of a round fall into a few bins: the lanes of a warp that hit
-        //  the same bin are counted by one of them, instead of 32 atomics on one shared-memory word)
-        for (int base = 0; base < V; base += ACC_THREADS) { // the same trip count for every thread
-            const int v = base + (int)threadIdx.x;
-            const unsigned key = v < V ? orderable(z[v]) : 0u;
-            const bool in = v < V && (key & himask) == prefix;
-            const unsigned bin = (key >> shift) & 255u;
+//
+// One selection round: among the keys that agree with s.sel_prefix on the bits above shift + bits, count how many fall into
+// each value of the next `bits` bits, find the digit that holds the s.sel_k-th largest of them, and narrow prefix and rank.
+// The digit is found by all threads (chunk sums, a scan over the block, then the owner of the chunk walks it), not by one
+// thread walking the histogram.  KeyAt(i) is the i-th key; `aggregate`: the lanes of a warp that hit the same bin are counted
+// by one of them (logits share their leading bits, so in the first rounds most keys of a warp fall into a few bins).
+constexpr int SEL_MAX_BITS = 11, SEL_CAND = 4096;
+template <class KeyAt>
+__device__ void select_round(KeyAt key_at, int count, int shift, int bits, bool aggregate, BlockScratch &s) {
+    const int tid = threadIdx.x, nbins = 1 << bits;
+    for (int b = tid; b < nbins; b += ACC_THREADS) s.hist[b] = 0u;
+    __syncthreads();
+    const unsigned prefix = s.sel_prefix, kk = s.sel_k;
+    const unsigned himask = (shift + bits >= 32) ? 0u : (0xffffffffu << (shift + bits));
+    const unsigned dmask = (unsigned)nbins - 1u;
+    for (int base = 0; base < count; base += ACC_THREADS) { // the same trip count for every thread
+        const int i = base + tid;
+        const unsigned key = i < count ? key_at(i) : 0u;
+        const bool in = i < count && (key & himask) == prefix;
+        const unsigned bin = (key >> shift) & dmask;
+        if (aggregate) {
             const unsigned voters = __ballot_sync(0xffffffffu, in);
             if (in) {
                 const unsigned peers = __match_any_sync(voters, bin);
-                if ((int)(threadIdx.x & 31) == __ffs(peers) - 1) atomicAdd(&s.hist[bin], (unsigned)__popc(peers));
+                if ((tid & 31) == __ffs(peers) - 1) atomicAdd(&s.hist[bin], (unsigned)__popc(peers));
             }
+        } else if (in) {
+            atomicAdd(&s.hist[bin], 1u);
         }
-        __syncthreads();
-        if (threadIdx.x == 0) {
-            unsigned cum = 0, kk = s.sel_k;
-            for (int b = 255; b >= 0; --b) {
-                if (cum + s.hist[b] >= kk) { s.sel_prefix = prefix | ((unsigned)b << shift); s.sel_k = kk - cum; break; }
-                cum += s.hist[b];
-            }
+    }
+    __syncthreads();
+    // bins in descending order, `per` consecutive ones per thread
+    const int per = (nbins + ACC_THREADS - 1) / ACC_THREADS, d0 = tid * per;
+    unsigned mine = 0;
+    for (int j = 0; j < per; ++j) { const int d = d0 + j; if (d < nbins) mine += s.hist[nbins - 1 - d]; }
+    unsigned incl = mine;
+#pragma unroll
+    for (int off = 1; off < 32; off <<= 1) {
+        const unsigned t = __shfl_up_sync(0xffffffffu, incl, off);
+        if ((tid & 31) >= off) incl += t;
+    }
+    if ((tid & 31) == 31) s.i[tid >> 5] = (int)incl;
+    __syncthreads();
+    unsigned before = 0;
+    for (int w = 0; w < (tid >> 5); ++w) before += (unsigned)s.i[w];
+    const unsigned excl = before + incl - mine;
+    __syncthreads(); // (s.i is free again, and nobody reads the old prefix after this point)
+    if (excl < kk && kk <= excl + mine) { // exactly one thread: the k-th largest lies in its chunk
+        unsigned cum = excl;
+        for (int j = 0; j < per; ++j) {
+            const int b = nbins - 1 - (d0 + j);
+            const unsigned h = s.hist[b];
+            if (cum + h >= kk) { s.sel_prefix = prefix | ((unsigned)b << shift); s.sel_k = kk - cum; break; }
+            cum += h;
         }
+    }
+    __syncthreads();
+}
+
+// Keys of the row that pass `keep` -> s.cand (in no particular order); returns how many there are (possibly more than fit).
+template <class Keep>
+__device__ int gather_keys(const float *__restrict__ z, int V, Keep keep, BlockScratch &s) {
+    const int tid = threadIdx.x;
+    if (tid == 0) s.flag = 0;
+    __syncthreads();
+    for (int base = 0; base < V; base += ACC_THREADS) {
+        const int v = base + tid;
+        const unsigned key = v < V ? orderable(z[v]) : 0u;
+        const bool in = v < V && keep(key);
+        const unsigned voters = __ballot_sync(0xffffffffu, in);
+        if (voters) {
+            int at = 0;
+            if ((tid & 31) == 0) at = atomicAdd(&s.flag, __popc(voters));
+            at = __shfl_sync(0xffffffffu, at, 0) + __popc(voters & ((1u << (tid & 31)) - 1u));
+            if (in && at < SEL_CAND) s.cand[at] = key;
+        }
+    }
+    __syncthreads();
+    const int n = s.flag;
+    __syncthreads();
+    return n;
+}
+// The k-th largest of the first `count` keys in s.cand: four rounds of eight bits.
+__device__ unsigned kth_of_cand(int count, int k, BlockScratch &s) {
+    if (threadIdx.x == 0) { s.sel_prefix = 0u; s.sel_k = (unsigned)k; }
+    __syncthreads();
+    const unsigned *cand = s.cand;
+    auto from_cand = [cand](int i) { return cand[i]; };
+    for (int shift = 24; shift >= 0; shift -= 8) select_round(from_cand, count, shift, 8, shift >= 16, s);
+    return s.sel_prefix;
+}
+
+// `my_max`: the largest logit among the ones this thread looked at in the pass before (thread t: z[t], z[t + ACC_THREADS], ...).
+// For k up to the number of threads, the k-th largest of those maxima is a lower bound of the k-th largest of the row - k
+// different entries are at least as large - so only the entries at or above it, usually a few times k, stay in the running:
+// they are gathered into shared memory in one pass over the row and the selection is finished there.  The histogram rounds
+// over the whole row are the general path (a larger k, or too many entries at or above the bound: ties, a narrow row): the
+// first round looks at the top 11 bits (sign, exponent, two fraction bits: a quarter of a binade per bin), the keys of the bin
+// the k-th largest falls into are gathered, and the remaining 21 bits are settled in shared memory; should more than SEL_CAND
+// keys share those 11 bits, the later rounds read the row again instead.  (Counting a whole row into a histogram in shared
+// memory is slow - 50 us for a GPT-2 vocabulary - because most logits fall into a few bins and the additions to one bin queue up.)
+__device__ float kth_largest(const float *__restrict__ z, int V, int k, BlockScratch &s, float my_max) {
+    const int tid = threadIdx.x;
+    if (k <= ACC_THREADS) {
         __syncthreads();
+        s.cand[tid] = orderable(my_max);
+        __syncthreads();
+        const unsigned bound = kth_of_cand(ACC_THREADS, k, s);
+        const int cands = gather_keys(z, V, [bound](unsigned key) { return key >= bound; }, s);
+        if (cands <= SEL_CAND) return from_orderable(kth_of_cand(cands, k, s));
+    }
+    if (tid == 0) { s.sel_prefix = 0u; s.sel_k = (unsigned)k; }
+    __syncthreads();
+    auto from_row = [z](int i) { return orderable(z[i]); };
+    select_round(from_row, V, 32 - SEL_MAX_BITS, SEL_MAX_BITS, true, s);
+    const unsigned top = s.sel_prefix >> (32 - SEL_MAX_BITS);
+    const int cands = gather_keys(z, V, [top](unsigned key) { return (key >> (32 - SEL_MAX_BITS)) == top; }, s);
+    const unsigned *cand = s.cand;
+    auto from_cand = [cand](int i) { return cand[i]; };
+    const int rounds[3][2] = {{13, 8}, {5, 8}, {0, 5}};
+    for (int r = 0; r < 3; ++r) {
+        if (cands <= SEL_CAND) select_round(from_cand, cands, rounds[r][0], rounds[r][1], false, s);
+        else select_round(from_row, V, rounds[r][0], rounds[r][1], true, s);
     }
     return from_orderable(s.sel_prefix);
 }
@@ -209,7 +304,7 @@ __device__ int row_law(const float *__restrict__ z, int V, double temperature, i
     for (int v = tid; v < V; v += ACC_THREADS) { const float zv = z[v]; bad |= !isfinite(zv); zmax = fmaxf(zmax, zv); }
     if (block_max_int(bad, s)) return 1;
     float thr = -INFINITY;
-    if (top_k > 0 && top_k < V) thr = kth_largest(z, V, top_k, s);
+    if (top_k > 0 && top_k < V) thr = kth_largest(z, V, top_k, s, zmax);
     // (x / 1.0 is x exactly: at temperature 1 the fp64 division, a large part of this function's time, is skipped)
     const bool unit_t = temperature == 1.0;
     const double zm = block_max((double)zmax, s);
@@ -234,28 +329,31 @@ __device__ int row_law(const float *__restrict__ z, int V, double temperature, i
 // With a top-k cut a row's law is positive at few indices: list them (ascending), so that the walk's residual updates
 // and its inverse-CDF scan touch those entries only instead of the whole vocabulary.
 __device__ void list_support(const double *__restrict__ r, int V, int32_t *__restrict__ idx, int32_t *__restrict__ cnt, BlockScratch &s) {
-    const int tid = threadIdx.x, chunk = (V + ACC_THREADS - 1) / ACC_THREADS;
-    const int v0 = min(V, tid * chunk), v1 = min(V, v0 + chunk);
+    // warp w lists its contiguous share of the row, its lanes reading consecutive entries (ascending order is kept: by
+    // iteration, then by lane); a first pass counts, a scan over the warps gives each its place, a second pass writes
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5, warps = ACC_THREADS / 32;
+    const int chunk = (V + warps - 1) / warps, v0 = min(V, warp * chunk), v1 = min(V, v0 + chunk);
     int mine = 0;
-    for (int v = v0; v < v1; ++v) mine += r[v] > 0.0;
-    int incl = mine; // inclusive scan over the block: warp, then warp totals
-#pragma unroll
-    for (int off = 1; off < 32; off <<= 1) {
-        const int t = __shfl_up_sync(0xffffffffu, incl, off);
-        if ((tid & 31) >= off) incl += t;
+    for (int base = v0; base < v1; base += 32) { // (the same trip count for the lanes of a warp)
+        const int v = base + lane;
+        mine += __popc(__ballot_sync(0xffffffffu, v < v1 && r[v] > 0.0));
     }
     __syncthreads();
-    if ((tid & 31) == 31) s.i[tid >> 5] = incl;
+    if (lane == 0) s.i[warp] = mine;
     __syncthreads();
-    int base = 0, total = 0;
-    for (int w = 0; w < ACC_THREADS / 32; ++w) {
-        if (w < (tid >> 5)) base += s.i[w];
+    int at = 0, total = 0;
+    for (int w = 0; w < warps; ++w) {
+        if (w < warp) at += s.i[w];
         total += s.i[w];
     }
     if (total <= SSD_ACC_SUPPORT) {
-        int at = base + incl - mine;
-        for (int v = v0; v < v1; ++v)
-            if (r[v] > 0.0) idx[at++] = v;
+        for (int base = v0; base < v1; base += 32) {
+            const int v = base + lane;
+            const bool pos = v < v1 && r[v] > 0.0;
+            const unsigned m = __ballot_sync(0xffffffffu, pos);
+            if (pos) idx[at + __popc(m & ((1u << lane) - 1u))] = v;
+            at += __popc(m);
+        }
     }
     if (tid == 0) *cnt = total <= SSD_ACC_SUPPORT ? total : -1;
     __syncthreads();

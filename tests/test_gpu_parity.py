@@ -217,7 +217,8 @@ def test_accept_special_rows(tiny):
 def test_sampling_at_a_large_vocabulary_star_tree_ties_and_long_support(ssd):
     """The sampling rule on hand-made logits at a 50257-word vocabulary (a context without weights is enough for
     acceptance): a star of 40 children (many refusals at one node), top-k cuts whose kept set is short, tied, and -
-    with 3000 logits tied at the k-th value - longer than the support list the kernel keeps per row."""
+    with 3000 logits tied at the k-th value - longer than the support list the kernel keeps per row; rows that send the
+    selection of the k-th largest down each of its paths; k = 1 and k = V - 1."""
     import torch
     cfg = ssd_synth.config("gpt2_small")
     V = cfg["vocab"]
@@ -232,9 +233,16 @@ def test_sampling_at_a_large_vocabulary_star_tree_ties_and_long_support(ssd):
         tied = logits.copy()
         tied[:, rng.choice(V, size=3000, replace=False)] = 9.0   # 3000 ties at the top: any k <= 3000 keeps them all
         draft = ssd_synth.draft_rows_gamma(n, V, rng)
-        lg_dev, tied_dev, dp_dev = (torch.from_numpy(a).cuda() for a in (logits, tied, draft))
+        # the k-th largest is found by radix selection, whose first round looks at a logit's top 11 bits and whose later rounds
+        # work on the logits sharing them if they are few: a row inside one quarter of a binade (all share them), and the same
+        # row negated (the order of the bit patterns turns round below zero)
+        narrow = rng.uniform(8.0, 9.99, size=(n, V)).astype(np.float32)
+        narrow[0, tokens[1:]] = 9.995
+        below = (-narrow).astype(np.float32)
+        lg_dev, tied_dev, dp_dev, narrow_dev, below_dev = (torch.from_numpy(a).cuda() for a in (logits, tied, draft, narrow, below))
         fragile = 0
-        for lg_np, lg_d, top_k in ((logits, lg_dev, 0), (logits, lg_dev, 50), (logits, lg_dev, 1000), (tied, tied_dev, 50), (tied, tied_dev, 0)):
+        for lg_np, lg_d, top_k in ((logits, lg_dev, 0), (logits, lg_dev, 50), (logits, lg_dev, 1000), (tied, tied_dev, 50), (tied, tied_dev, 0),
+                                   (narrow, narrow_dev, 50), (narrow, narrow_dev, 5000), (below, below_dev, 50), (logits, lg_dev, 1), (logits, lg_dev, V - 1)):
             for step in range(3):
                 srng = ssd.binding.ssd_rng(5, step)
                 got = ctx.accept_tree(lg_d.data_ptr(), dp_dev.data_ptr(), tokens, parent, mode=ssd.SSD_SAMPLING, temperature=1.0,
