@@ -373,6 +373,17 @@ def per_kernel_roofline(run: Runner, parent, tokens, peak_gbs):
     out["layer_us"] = float((deps[-1] - deps[2]) / (L - 3) / 1e3)
     out["how"] = ("device timer stamps taken inside the kernels of one traced forward (dependencies met -> latest CTA end), "
                   "median over layers; tracing itself slows the forward by a few percent")
+    # The chain itself: from one kernel's dependencies being met to the next one's (median over layers), and one middle layer's
+    # stamps relative to its first kernel's dependencies (first CTA: entry, dependencies met, first accumulator complete - the
+    # projections only - and end; then the latest end over all CTAs).
+    flat = np.concatenate([body[:, :, 1].reshape(-1), [t[setup + per * L, 1]]]).astype(np.float64)
+    step = np.diff(flat).reshape(L, per)
+    out["phase_us"] = {name: float(v) for name, v in zip(names, np.median(step[2:], axis=0) / 1e3)}
+    mid = body[L // 2]
+    t0 = mid[0, 1]
+    rel = lambda v: None if v == 0 else round(float(v - t0) / 1e3, 2)
+    out["timeline_us"] = {"layer": L // 2, "columns": ["entry", "dependencies_met", "accumulator", "end", "latest_end"],
+                          "rows": {name: [rel(r[0]), rel(r[1]), rel(r[3]), rel(r[2]), rel(r[6])] for name, r in zip(names, mid)}}
     return out
 
 
