@@ -242,6 +242,9 @@ gemm_ws_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant_
             int seg = 0;
             bool ok = true;
             int kt = u0 % p.k_tiles, s = 0, round = 0; // (kept incrementally: no integer division inside the loop)
+            // (no stage can be complete before the previous kernel has produced the activations: wait for that in hardware rather
+            //  than by polling the first stage's barrier next to the CTAs that are still at work on this SM)
+            ptx::pdl_grid_wait();
             for (int u = u0; u < u1 && ok; ++u) {
                 const int j = u - u0;
                 const bool seg_first = (u == u0) || (kt == 0);
