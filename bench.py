@@ -46,9 +46,10 @@ METRIC = "GPT-2-L-shape tree-verify us/step (verify+accept+commit)"
 UNIT = "us/step"
 NOMINAL_HBM_GBS = 8000.0
 PLANT_PROBABILITY = 0.6
-# DRAM bytes (read + write) of one forward of the metric's workload: sum over the ncu launch list in
-# profiles/bench_step_gpt2_large_n32_launch_list.md (per forward, like `achieved`)
-NCU_TRAFFIC_BYTES = {("gpt2_large", 32, 256): 1758.2e6}
+# DRAM bytes (read + write) of one forward: sums over the forward's kernels in the ncu launch lists under profiles/
+# (bench_step_gpt2_large_n32_launch_list.md - a later capture of the same forward, in the sampling list, gives 1760.7 MB -
+# and bench_step_gpt2_large_n256_launch_list.md); per forward, like `achieved`
+NCU_TRAFFIC_BYTES = {("gpt2_large", 32, 256): 1758.2e6, ("gpt2_large", 256, 256): 2894.2e6}
 
 
 def measured_peaks():
