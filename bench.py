@@ -564,6 +564,71 @@ def run_staged(args, local, peaks, alphas=(0.3, 0.6, 0.9), n_tokens=256):
     return out
 
 
+def run_staged_decoder(local, n_tokens=192, prompt_len=64, table_tokens=320):
+    """The three-stage loop itself (target <- draft <- trigram table) through the public API, set up so that all three stages
+    contribute tokens although the weights are random: the GPT-2-small-shaped model is the target AND its own draft, decoding is
+    deterministic, and the trigram table is built from the model's own continuation of the prompt (as the paper builds its
+    table from samples of the draft).  Reports which stage every emitted token came from, tokens per target forward and the
+    loop's tokens/s (host bookkeeping of the loop included), and whether the output equals plain one-token-at-a-time decoding."""
+    import torch
+    import paper_2308_04623_b200 as ssd
+    from paper_2308_04623_b200.staged import StagedDecoder
+    cfg = ssd_synth.config("gpt2_small")
+    V = cfg["vocab"]
+    bits = ssd_synth.bf16_bits(ssd_synth.make_weights(cfg, seed=11))
+    stream = torch.cuda.current_stream()
+    c0 = ssd.Context(cfg, device=local, stream=stream.cuda_stream)
+    c1 = ssd.Context(cfg, device=local, stream=stream.cuda_stream)
+    c0.load_weights(bits)
+    c1.load_weights(bits)
+    prompt = [int(t) for t in ssd_synth.uniform_tokens(prompt_len, V, np.random.default_rng(12))]
+    # plain decoding: one node per forward
+    kv = c0.new_kv()
+    buf = torch.empty((64, V), dtype=torch.float32, device="cuda")
+    body = np.asarray(prompt[:-1], dtype=np.int32)
+    c0.verify_tree(body, ssd_synth.tree_chain(len(body)), kv, buf.data_ptr())
+    c0.kv_commit(kv, np.arange(len(body), dtype=np.int32))
+    plain, tok = [], prompt[-1]
+    one, root_only = np.zeros(1, dtype=np.int32), np.array([-1], dtype=np.int32)
+    p0, p1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    for i in range(table_tokens):
+        if i == 32:   # (the first steps carry the graph capture of the one-node forward)
+            p0.record(stream)
+        one[0] = tok
+        c0.verify_tree(one, root_only, kv, buf.data_ptr())
+        c0.kv_commit(kv, np.zeros(1, dtype=np.int32))
+        tok = int(torch.argmax(buf[0]).item())
+        plain.append(tok)
+    p1.record(stream)
+    torch.cuda.synchronize()
+    plain_tok_s = (table_tokens - 32) / (p0.elapsed_time(p1) * 1e-3)
+    kv.close()
+    tri = ssd.Trigram(np.asarray(prompt + plain, dtype=np.int32), V, device=local, stream=stream.cuda_stream)
+    res = None
+    for timed in (False, True):   # (an untimed pass first: graph captures and first launches)
+        dec = StagedDecoder(c0, c1, tri, mode=ssd.SSD_GREEDY, rounds=2, siblings=1, seed=3)
+        dec.prefill(prompt)
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record(stream)
+        got = dec.generate(n_tokens if timed else 24)
+        e1.record(stream)
+        torch.cuda.synchronize()
+        if timed:
+            ms = e0.elapsed_time(e1)
+            st = dec.stats
+            res = {"emitted_tokens": len(got), "target_forwards": st["target_steps"], "draft_forwards": st["draft_forwards"],
+                   "tokens_per_target_forward": st["emitted"] / max(1, st["target_steps"]), "tokens_per_s": len(got) / (ms * 1e-3),
+                   "token_origin": dict(st["origin"]), "equals_plain_decoding": got == plain[:len(got)],
+                   "plain_decoding_tokens_per_s": plain_tok_s,
+                   "note": "GPT-2-small-shaped random weights as target and as its own draft, deterministic decoding, trigram table "
+                           "built from the model's own continuation of the 64-token prompt; the loop's host bookkeeping is inside the time"}
+        dec.close()
+    tri.close()
+    c0.close()
+    c1.close()
+    return res
+
+
 def run_gpu(args):
     import torch
 
@@ -649,6 +714,7 @@ def run_gpu(args):
             del r2
         sweep.update(run_sweep(args, local, peaks))
         sweep["config4"] = run_staged(args, local, peaks)
+        sweep["config4"]["staged_decoder_self_draft"] = run_staged_decoder(local)
         sweep["w8"] = run_w8(args, local, peaks)
         line["sweep"] = sweep
     if world == 1 and not args.no_cpu_baseline:
