@@ -278,6 +278,10 @@ int ssd_kv_read(ssd_ctx *ctx, const ssd_kv *kv, int32_t layer, int32_t which, in
  *   SSD_TUNE_STAGE_KV_FROM [128]  bf16 models: trees of at least this many nodes get one more kernel per layer, which writes the tree's
  *                                 K / V rows to the cache's scratch slots so that the attention reads every key block from the cache
  *                                 (otherwise each 16-node tile of a head converts and stages the whole tree's keys itself); 0 = never
+ *                                 (whatever the value, other than 0, trees of 64 nodes or more also take that path when heads x 16-node
+ *                                 tiles exceed the SM count: the self-staging CTAs, one per SM, would run in two waves)
+ *   SSD_TUNE_ATTN_STAGED_WARPS [0] warps of an attention CTA on that path: 4 (three CTAs per SM), 8 (two per SM, half as many key blocks per
+ *                                 warp); 0 = eight when two CTAs per SM hold every (head, 16-node tile) at once, else four
  *   SSD_TUNE_ATTN_SPLITS [0]      bf16 models: CTAs (one thread-block cluster) that share a (head, 16-node tile) of the attention, each
  *                                 with a part of the keys, merged in the first one's shared memory: 1, 2 or 4; 0 = from the prefix
  *                                 length of each call (1 up to 19 key blocks of 16, 2 up to 27, else 4)
@@ -291,7 +295,7 @@ int ssd_kv_read(ssd_ctx *ctx, const ssd_kv *kv, int32_t layer, int32_t which, in
  */
 enum { SSD_TUNE_LOW_PLANE = 0, SSD_TUNE_DEPENDENT_LAUNCH = 1, SSD_TUNE_GRAPH = 2, SSD_TUNE_GEMM_CTAS = 3, SSD_TUNE_CLUSTER_REDUCE = 4,
        SSD_TUNE_CLUSTER_MAX = 5, SSD_TUNE_ATTN_LOW_PLANE = 6, SSD_TUNE_HEAD_CTAS = 7, SSD_TUNE_KERNEL_TRACE = 8, SSD_TUNE_CLUSTER_QKV = 9, SSD_TUNE_CLUSTER_O = 10,
-       SSD_TUNE_CLUSTER_FC = 11, SSD_TUNE_CLUSTER_PROJ = 12, SSD_TUNE_HEAD_STATS = 13, SSD_TUNE_W8_PLANES = 14, SSD_TUNE_STAGE_KV_FROM = 15, SSD_TUNE_ATTN_SPLITS = 16, SSD_TUNE_NODE_GROUPS = 17, SSD_TUNE_FUSED_GELU = 18 };
+       SSD_TUNE_CLUSTER_FC = 11, SSD_TUNE_CLUSTER_PROJ = 12, SSD_TUNE_HEAD_STATS = 13, SSD_TUNE_W8_PLANES = 14, SSD_TUNE_STAGE_KV_FROM = 15, SSD_TUNE_ATTN_SPLITS = 16, SSD_TUNE_NODE_GROUPS = 17, SSD_TUNE_FUSED_GELU = 18, SSD_TUNE_ATTN_STAGED_WARPS = 19 };
 int ssd_set_tuning(ssd_ctx *ctx, int32_t knob, int32_t value);
 
 /*

@@ -16,7 +16,7 @@ SSD_DTYPE_F32, SSD_DTYPE_BF16, SSD_DTYPE_BF16_W8 = 0, 1, 2
 SSD_TUNE_LOW_PLANE, SSD_TUNE_DEPENDENT_LAUNCH, SSD_TUNE_GRAPH, SSD_TUNE_GEMM_CTAS, SSD_TUNE_CLUSTER_REDUCE, SSD_TUNE_CLUSTER_MAX = 0, 1, 2, 3, 4, 5
 SSD_TUNE_ATTN_LOW_PLANE, SSD_TUNE_HEAD_CTAS, SSD_TUNE_KERNEL_TRACE = 6, 7, 8
 SSD_TUNE_CLUSTER_QKV, SSD_TUNE_CLUSTER_O, SSD_TUNE_CLUSTER_FC, SSD_TUNE_CLUSTER_PROJ, SSD_TUNE_HEAD_STATS = 9, 10, 11, 12, 13
-SSD_TUNE_W8_PLANES, SSD_TUNE_STAGE_KV_FROM, SSD_TUNE_ATTN_SPLITS, SSD_TUNE_NODE_GROUPS, SSD_TUNE_FUSED_GELU = 14, 15, 16, 17, 18
+SSD_TUNE_W8_PLANES, SSD_TUNE_STAGE_KV_FROM, SSD_TUNE_ATTN_SPLITS, SSD_TUNE_NODE_GROUPS, SSD_TUNE_FUSED_GELU, SSD_TUNE_ATTN_STAGED_WARPS = 14, 15, 16, 17, 18, 19
 
 # every symbol include/ssd.h declares
 EXPORTS = ("ssd_create", "ssd_load_weights", "ssd_w8_read", "ssd_kv_create", "ssd_kv_reset", "ssd_kv_len", "ssd_kv_rollback",

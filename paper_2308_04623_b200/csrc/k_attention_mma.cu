@@ -7,7 +7,8 @@ namespace {
 // blocks and multiplies masked keys' V by zero weights).  One CTA of 128 threads per (head, 16 slots).
 // V is written as 16-byte groups of eight consecutive slots of one dimension, aligned in the cache row: a group that begins below
 // kv_len keeps the committed values it holds (read, merged, written back by the one thread that owns the group).
-constexpr int NW_STAGED = 4; // warps of an attention CTA that reads every block from the cache: three such CTAs share an SM
+constexpr int NW_STAGED = 4; // warps of an attention CTA that reads every block from the cache: three such CTAs share an SM ...
+constexpr int NW_STAGED_WIDE = 8; // ... or eight, two CTAs per SM, when that many slots hold all (head, node tile) items at once
 __global__ void __launch_bounds__(128)
 kv_stage_kernel(const float *__restrict__ qkv, const StepInfo *__restrict__ info, size_t layer_offset, int n, int d, int cap, unsigned long long *trace) {
     if (threadIdx.x == 0) ptx::trace_mark(trace, 0);
@@ -47,8 +48,9 @@ kv_stage_kernel(const float *__restrict__ qkv, const StepInfo *__restrict__ info
     if (trace) { __syncthreads(); if (threadIdx.x == 0) ptx::trace_mark(trace, 2); }
 }
 
-template <bool LO, bool STAGED>
-__global__ void __maxnreg__(144)
+// STAGED: 0 = the CTA converts and stages the tree's keys itself (NW_MAX warps); otherwise the warps of a CTA that reads them from the cache
+template <bool LO, int STAGED>
+__global__ void __maxnreg__((STAGED == NW_STAGED_WIDE ? 128 : 144))
 tree_attention_mma_kernel(const float *__restrict__ qkv, const StepInfo *__restrict__ info, size_t layer_offset, TreeMeta meta, int n, int d,
                           int cap, __nv_bfloat16 *__restrict__ o_hi, __nv_bfloat16 *__restrict__ o_lo, unsigned long long *trace,
                           uint8_t *__restrict__ planes8, size_t plane_stride) {
@@ -61,7 +63,7 @@ tree_attention_mma_kernel(const float *__restrict__ qkv, const StepInfo *__restr
     attn::Output out = {o_hi, o_lo, nullptr, nullptr, 0, 0, splits > 1 ? 1 : 0, planes8, plane_stride};
     // (the step's tree metadata and the committed cache rows were complete before the first dependent launch of the
     //  forward began, so the item reads them before it waits for the QKV projection)
-    attn::work_item<(STAGED ? NW_STAGED : attn::NW_MAX), true, true, LO, STAGED>(threadIdx.x, 0, smem_raw, blockIdx.x, blockIdx.y * 16, split, splits,
+    attn::work_item<(STAGED ? STAGED : attn::NW_MAX), true, true, LO, (STAGED != 0)>(threadIdx.x, 0, smem_raw, blockIdx.x, blockIdx.y * 16, split, splits,
                                                                                  blockIdx.y == 0 && split == splits - 1, qkv, info, layer_offset, meta, n, d, cap, out, trace);
     if (trace) { __syncthreads(); if (threadIdx.x == 0) ptx::trace_mark(trace, 2); }
 }
@@ -71,8 +73,9 @@ size_t tree_attention_mma_smem(int n) { return attn::smem_bytes(n); }
 
 cudaError_t tree_attention_mma_prepare() {
     cudaError_t e = cudaSuccess;
-    const void *kernels[] = {(const void *)tree_attention_mma_kernel<true, false>, (const void *)tree_attention_mma_kernel<false, false>,
-                             (const void *)tree_attention_mma_kernel<true, true>, (const void *)tree_attention_mma_kernel<false, true>};
+    const void *kernels[] = {(const void *)tree_attention_mma_kernel<true, 0>, (const void *)tree_attention_mma_kernel<false, 0>,
+                             (const void *)tree_attention_mma_kernel<true, NW_STAGED>, (const void *)tree_attention_mma_kernel<false, NW_STAGED>,
+                             (const void *)tree_attention_mma_kernel<true, NW_STAGED_WIDE>, (const void *)tree_attention_mma_kernel<false, NW_STAGED_WIDE>};
     for (const void *k : kernels) {
         if (e == cudaSuccess) e = cudaFuncSetAttribute(k, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)attn::smem_bytes(SSD_MAX_NODES, attn::NW_MAX, false, 8));
         if (e == cudaSuccess) e = cudaFuncSetAttribute(k, cudaFuncAttributePreferredSharedMemoryCarveout, cudaSharedmemCarveoutMaxShared);
@@ -97,12 +100,15 @@ cudaError_t launch_kv_stage(const float *qkv, const StepInfo *info, size_t layer
 
 cudaError_t launch_tree_attention_mma(const float *qkv, const StepInfo *info, size_t layer_offset_elems, const TreeMeta &m, int n, int n_head,
                                       int cap, __nv_bfloat16 *o_hi, __nv_bfloat16 *o_lo, bool pdl, cudaStream_t s, unsigned long long *trace, bool lo_pairs,
-                                      uint8_t *planes8, size_t plane_stride, bool staged, int splits) {
+                                      uint8_t *planes8, size_t plane_stride, bool staged, int splits, int sm_count) {
     if (splits < 1 || splits > 8 || (staged && splits != 1)) return cudaErrorInvalidValue;
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3(n_head, (n + 15) / 16, splits);
-    cfg.blockDim = dim3((staged ? NW_STAGED : attn::NW_MAX) * 32);
-    cfg.dynamicSmemBytes = attn::smem_bytes(n, staged ? NW_STAGED : attn::NW_MAX, staged, splits);
+    // (reading from the cache: eight warps - half as many key blocks per warp - if two such CTAs per SM hold every item at once)
+    const int tiles = (n + 15) / 16;
+    const int nw = !staged ? attn::NW_MAX : (sm_count > 0 && n_head * tiles <= 2 * sm_count) ? NW_STAGED_WIDE : NW_STAGED;
+    cfg.blockDim = dim3(nw * 32);
+    cfg.dynamicSmemBytes = attn::smem_bytes(n, nw, staged, splits);
     cfg.stream = s;
     cudaLaunchAttribute attr[2];
     int na = 0;
@@ -118,7 +124,8 @@ cudaError_t launch_tree_attention_mma(const float *qkv, const StepInfo *info, si
     }
     cfg.attrs = attr;
     cfg.numAttrs = na;
-    auto kernel = staged ? (lo_pairs ? tree_attention_mma_kernel<true, true> : tree_attention_mma_kernel<false, true>)
-                         : (lo_pairs ? tree_attention_mma_kernel<true, false> : tree_attention_mma_kernel<false, false>);
+    auto kernel = nw == NW_STAGED_WIDE ? (lo_pairs ? tree_attention_mma_kernel<true, NW_STAGED_WIDE> : tree_attention_mma_kernel<false, NW_STAGED_WIDE>)
+                  : staged         ? (lo_pairs ? tree_attention_mma_kernel<true, NW_STAGED> : tree_attention_mma_kernel<false, NW_STAGED>)
+                                   : (lo_pairs ? tree_attention_mma_kernel<true, 0> : tree_attention_mma_kernel<false, 0>);
     return cudaLaunchKernelEx(&cfg, kernel, qkv, info, layer_offset_elems, m, n, n_head * attn::DH, cap, o_hi, o_lo, trace, planes8, plane_stride);
 }

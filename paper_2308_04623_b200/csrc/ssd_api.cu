@@ -64,6 +64,7 @@ struct ssd_ctx {
     struct ForwardGraph { cudaGraph_t graph; cudaGraphExec_t exec; cudaGraphNode_t prep_node; int kernels; };
     ForwardGraph graphs[SSD_MAX_NODES + 1][3]; // (second index: the attention's key splits, 1 / 2 / 4 - chosen from the prefix length at each call)
     int attn_splits;                           // 0 = choose; 1, 2, 4 = always that many
+    int attn_staged_warps;                     // 0 = choose; 4 or 8: warps of the attention CTAs that read the tree's rows from the cache
     int fused_gelu;                            // the back-projection makes its gelu(.) operand planes itself (no separate kernel)
     int node_groups;                           // trees of more than 64 nodes: the layers' projections run on node groups of 64
     cudaStream_t capture_stream;
@@ -221,9 +222,17 @@ static unsigned long long *trace_slot(ssd_ctx *ctx, int kernels) {
 // they all fit the GPU at once, and not on the large-tree path.  Measured (verify, us): GPT-2-small shape, prefix 512, 8 nodes:
 // 322 / 309 / 302 with 1 / 2 / 4 splits; GPT-2-XL shape, prefix 960, 8 nodes: 1993 / 1864 / 1705; prefix 512, 32 nodes: 1799 / 1763 /
 // 1979 (200 CTAs: two waves); GPT-2-large shape, prefix 256, 32 nodes (18 key blocks): 1057 / 1096.
+// Whether a tree's K / V rows go to the cache in a kernel of their own and the attention reads them from there: from
+// SSD_TUNE_STAGE_KV_FROM nodes on, and - with 64 nodes or more - as soon as there are more (head, node tile) items than SMs
+// (a CTA that stages the tree's rows itself has an SM to itself, so those items would run in two waves; measured at the
+// GPT-2-XL shape, 96 nodes = 150 items: 2875 against 2990 us per verify).
+static bool attn_staged(const ssd_ctx *ctx, int n) {
+    if (ctx->stage_kv_from <= 0) return false;
+    return n >= ctx->stage_kv_from || (n >= 64 && ctx->cfg.n_head * ((n + 15) / 16) > ctx->sm_count);
+}
 static int attn_splits_for(const ssd_ctx *ctx, int kv_len, int n) {
     const int tiles = (n + 15) / 16, ctas = ctx->cfg.n_head * tiles;
-    const bool staged = ctx->stage_kv_from > 0 && n >= ctx->stage_kv_from;
+    const bool staged = attn_staged(ctx, n);
     int s = ctx->attn_splits;
     if (s == 0) {
         const int blocks = (kv_len + n + 15) / 16;
@@ -307,7 +316,9 @@ cudaError_t enqueue_forward(ssd_ctx *ctx, int n, int cap, const NodeList &tk, co
         __nv_bfloat16 *a_lo = lo ? ctx->a_lo : nullptr, *o_lo = lo ? ctx->o_lo : nullptr, *h_lo = lo ? ctx->h_lo : nullptr;
         // Large trees: one small kernel per layer writes the tree's K / V rows to the cache's scratch slots and the attention reads
         // every key block from there, instead of each of a head's node tiles converting and staging the whole tree's keys itself.
-        const bool staged = ctx->stage_kv_from > 0 && n >= ctx->stage_kv_from;
+        const bool staged = attn_staged(ctx, n);
+        // (the launcher takes eight warps when heads x tiles fit 2 x this many slots: 0 forces four, a huge count eight)
+        const int attn_sms = ctx->attn_staged_warps == 4 ? 0 : ctx->attn_staged_warps == 8 ? (1 << 20) : sms;
         if (ctx->w8) {
             // 8-bit weights: the same eight launches per layer; the element-wise kernels and the attention write four e4m3 planes,
             // the projections run on the 8-bit tensor-core kind.  A CTA takes at most 128 nodes (512 accumulator columns); trees of
@@ -328,7 +339,7 @@ cudaError_t enqueue_forward(ssd_ctx *ctx, int n, int cap, const NodeList &tk, co
                 Q(launch_ln_prep(ctx->x, L.ln1_g, L.ln1_b, n, d, c.ln_eps, nullptr, nullptr, ctx->qkv, 3 * d, info, 0, pdl, s, trace_slot(ctx, *kernels), ctx->a8, sa));
                 Q(gemm8(&t[0], &ssd_ctx::ActMaps::a_hi, ctx->qkv, 3 * d, L.b_qkv, d, 3 * d, grid8, L.s_qkv));
                 if (staged) Q(launch_kv_stage(ctx->qkv, info, l * layer_elems, n, c.n_head, cap, pdl, s, trace_slot(ctx, *kernels)));
-                Q(launch_tree_attention_mma(ctx->qkv, info, l * layer_elems, ctx->meta, n, c.n_head, cap, nullptr, nullptr, pdl, s, trace_slot(ctx, *kernels), ctx->attn_lo != 0, ctx->o8, sa, staged, attn_splits));
+                Q(launch_tree_attention_mma(ctx->qkv, info, l * layer_elems, ctx->meta, n, c.n_head, cap, nullptr, nullptr, pdl, s, trace_slot(ctx, *kernels), ctx->attn_lo != 0, ctx->o8, sa, staged, attn_splits, attn_sms));
                 Q(gemm8(&t[1], &ssd_ctx::ActMaps::o_hi, ctx->x, d, L.b_o, d, d, grid8, L.s_o));
                 Q(launch_ln_prep(ctx->x, L.ln2_g, L.ln2_b, n, d, c.ln_eps, nullptr, nullptr, ctx->h, F, info, 0, pdl, s, trace_slot(ctx, *kernels), ctx->a8, sa));
                 Q(gemm8(&t[2], &ssd_ctx::ActMaps::a_hi, ctx->h, F, L.b_fc, d, F, grid8, L.s_fc));
@@ -366,7 +377,7 @@ cudaError_t enqueue_forward(ssd_ctx *ctx, int n, int cap, const NodeList &tk, co
             Q(launch_ln_prep(ctx->x, L.ln1_g, L.ln1_b, n, d, c.ln_eps, ctx->a_hi, a_lo, ctx->qkv, 3 * d, info, 0, pdl, s, trace_slot(ctx, *kernels)));
             Q(launch_gemm_ws(&t[0], &ag->a_hi, &ag->a_pair, ctx->qkv, info, 3 * d, L.b_qkv, n, d, 3 * d, lo, lgrid, sms, ctx->d_status, pdl, s, trace_slot(ctx, *kernels), nullptr, nullptr, 0, 4, gr));
             if (staged) Q(launch_kv_stage(ctx->qkv, info, l * layer_elems, n, c.n_head, cap, pdl, s, trace_slot(ctx, *kernels)));
-            Q(launch_tree_attention_mma(ctx->qkv, info, l * layer_elems, ctx->meta, n, c.n_head, cap, ctx->o_hi, o_lo, pdl, s, trace_slot(ctx, *kernels), ctx->attn_lo != 0, nullptr, 0, staged, attn_splits));
+            Q(launch_tree_attention_mma(ctx->qkv, info, l * layer_elems, ctx->meta, n, c.n_head, cap, ctx->o_hi, o_lo, pdl, s, trace_slot(ctx, *kernels), ctx->attn_lo != 0, nullptr, 0, staged, attn_splits, attn_sms));
             Q(launch_gemm_ws(&t[1], &ag->o_hi, &ag->o_pair, ctx->x, info, d, L.b_o, n, d, d, lo, lgrid, sms, ctx->d_status, pdl, s, trace_slot(ctx, *kernels), nullptr, nullptr, 0, 4, gr));
             Q(launch_ln_prep(ctx->x, L.ln2_g, L.ln2_b, n, d, c.ln_eps, ctx->a_hi, a_lo, ctx->h, F, info, 0, pdl, s, trace_slot(ctx, *kernels)));
             Q(launch_gemm_ws(&t[2], &af->a_hi, &af->a_pair, ctx->h, info, F, L.b_fc, n, d, F, lo, lgrid, sms, ctx->d_status, pdl, s, trace_slot(ctx, *kernels), nullptr, nullptr, 0, 4, gr_fc));
@@ -500,6 +511,7 @@ int ssd_create(const ssd_config *cfg, int device, void *cuda_stream, ssd_ctx **o
     ctx->attn_splits = 0;
     ctx->node_groups = 1;
     ctx->fused_gelu = 0;
+    ctx->attn_staged_warps = 0;
     ctx->stage_kv_from = 128; // (measured at the GPT-2-large shape: 2 % faster at 128 nodes, 14 % at 256, slower below)
     ctx->device = device;
     ctx->stream = (cudaStream_t)cuda_stream;
@@ -1033,6 +1045,7 @@ int ssd_set_tuning(ssd_ctx *ctx, int32_t knob, int32_t value) {
     case SSD_TUNE_HEAD_STATS: if (value != 0 && value != 1) return SSD_ERR_BAD_ARG; ctx->use_head_stats = value; ctx->head_logits = nullptr; break;
     case SSD_TUNE_STAGE_KV_FROM: if (value < 0 || value > SSD_MAX_NODES + 1) return SSD_ERR_BAD_ARG; ctx->stage_kv_from = value; break;
     case SSD_TUNE_NODE_GROUPS: if (value != 0 && value != 1) return SSD_ERR_BAD_ARG; ctx->node_groups = value; break;
+    case SSD_TUNE_ATTN_STAGED_WARPS: if (value != 0 && value != 4 && value != 8) return SSD_ERR_BAD_ARG; ctx->attn_staged_warps = value; break;
     case SSD_TUNE_FUSED_GELU: if (value != 0 && value != 1) return SSD_ERR_BAD_ARG; ctx->fused_gelu = value; break;
     case SSD_TUNE_ATTN_SPLITS: if (value != 0 && value != 1 && value != 2 && value != 4) return SSD_ERR_BAD_ARG; ctx->attn_splits = value; break;
     case SSD_TUNE_W8_PLANES:

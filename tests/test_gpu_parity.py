@@ -843,14 +843,16 @@ def test_w8_plane_count(ssd, util):
     p16.close()
 
 
-@pytest.mark.parametrize("prefix", [0, 5, 16, 37])
-def test_tree_rows_read_from_the_cache_give_the_same_logits(ssd, util, prefix):
+@pytest.mark.parametrize("prefix,warps", [(0, 4), (5, 8), (16, 4), (37, 8), (37, 4), (16, 8)])
+def test_tree_rows_read_from_the_cache_give_the_same_logits(ssd, util, prefix, warps):
     """Large trees: a kernel of its own writes the tree's K / V rows to the cache's scratch slots (and zeroes the rest of the last
     16-key block) and the attention reads every block from the cache.  Against the oracle and against the path in which every
     node tile stages the tree's keys itself, for prefixes that end on and off a 16-key boundary, with commits in between (the
-    scratch rows then become committed ones); forcing the path on a small tree covers the case of a single partial block."""
+    scratch rows then become committed ones); forcing the path on a small tree covers the case of a single partial block.  Both
+    shapes of the cache-reading CTA: four warps, and eight (the choice depends on how many (head, tile) items the GPU holds)."""
     rng = np.random.default_rng(61 + prefix)
     p = util.Pair("ragged_bf16", seed=3, qk_gain=3.0)
+    p.ctx.set_tuning(ssd.SSD_TUNE_ATTN_STAGED_WARPS, warps)
     V, L = p.V, p.cfg["n_layer"]
     if prefix:
         p.prefill(ssd_synth.uniform_tokens(prefix, V, rng))
