@@ -8,6 +8,7 @@ namespace {
 // V is written as 16-byte groups of eight consecutive slots of one dimension, aligned in the cache row: a group that begins below
 // kv_len keeps the committed values it holds (read, merged, written back by the one thread that owns the group).
 constexpr int NW_STAGED = 4; // warps of an attention CTA that reads every block from the cache: three such CTAs share an SM ...
+// (six warps at 112 registers per thread, still three CTAs per SM, were measured much slower: 3210 against 2547 us per verify of 256 nodes)
 constexpr int NW_STAGED_WIDE = 8; // ... or eight, two CTAs per SM, when that many slots hold all (head, node tile) items at once
 __global__ void __launch_bounds__(128)
 kv_stage_kernel(const float *__restrict__ qkv, const StepInfo *__restrict__ info, size_t layer_offset, int n, int d, int cap, unsigned long long *trace) {
@@ -100,13 +101,13 @@ cudaError_t launch_kv_stage(const float *qkv, const StepInfo *info, size_t layer
 
 cudaError_t launch_tree_attention_mma(const float *qkv, const StepInfo *info, size_t layer_offset_elems, const TreeMeta &m, int n, int n_head,
                                       int cap, __nv_bfloat16 *o_hi, __nv_bfloat16 *o_lo, bool pdl, cudaStream_t s, unsigned long long *trace, bool lo_pairs,
-                                      uint8_t *planes8, size_t plane_stride, bool staged, int splits, int sm_count) {
+                                      uint8_t *planes8, size_t plane_stride, int staged_warps, int splits) {
+    const bool staged = staged_warps != 0;
     if (splits < 1 || splits > 8 || (staged && splits != 1)) return cudaErrorInvalidValue;
+    if (staged && staged_warps != NW_STAGED && staged_warps != NW_STAGED_WIDE) return cudaErrorInvalidValue;
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3(n_head, (n + 15) / 16, splits);
-    // (reading from the cache: eight warps - half as many key blocks per warp - if two such CTAs per SM hold every item at once)
-    const int tiles = (n + 15) / 16;
-    const int nw = !staged ? attn::NW_MAX : (sm_count > 0 && n_head * tiles <= 2 * sm_count) ? NW_STAGED_WIDE : NW_STAGED;
+    const int nw = staged ? staged_warps : attn::NW_MAX;
     cfg.blockDim = dim3(nw * 32);
     cfg.dynamicSmemBytes = attn::smem_bytes(n, nw, staged, splits);
     cfg.stream = s;

@@ -317,8 +317,9 @@ cudaError_t enqueue_forward(ssd_ctx *ctx, int n, int cap, const NodeList &tk, co
         // Large trees: one small kernel per layer writes the tree's K / V rows to the cache's scratch slots and the attention reads
         // every key block from there, instead of each of a head's node tiles converting and staging the whole tree's keys itself.
         const bool staged = attn_staged(ctx, n);
-        // (the launcher takes eight warps when heads x tiles fit 2 x this many slots: 0 forces four, a huge count eight)
-        const int attn_sms = ctx->attn_staged_warps == 4 ? 0 : ctx->attn_staged_warps == 8 ? (1 << 20) : sms;
+        // (reading from the cache: eight warps per CTA - half as many key blocks per warp - if two such CTAs per SM hold every
+        //  (head, node tile) item at once, else four, three CTAs per SM)
+        const int attn_warps = !staged ? 0 : ctx->attn_staged_warps ? ctx->attn_staged_warps : c.n_head * ((n + 15) / 16) <= 2 * sms ? 8 : 4;
         if (ctx->w8) {
             // 8-bit weights: the same eight launches per layer; the element-wise kernels and the attention write four e4m3 planes,
             // the projections run on the 8-bit tensor-core kind.  A CTA takes at most 128 nodes (512 accumulator columns); trees of
@@ -339,7 +340,7 @@ cudaError_t enqueue_forward(ssd_ctx *ctx, int n, int cap, const NodeList &tk, co
                 Q(launch_ln_prep(ctx->x, L.ln1_g, L.ln1_b, n, d, c.ln_eps, nullptr, nullptr, ctx->qkv, 3 * d, info, 0, pdl, s, trace_slot(ctx, *kernels), ctx->a8, sa));
                 Q(gemm8(&t[0], &ssd_ctx::ActMaps::a_hi, ctx->qkv, 3 * d, L.b_qkv, d, 3 * d, grid8, L.s_qkv));
                 if (staged) Q(launch_kv_stage(ctx->qkv, info, l * layer_elems, n, c.n_head, cap, pdl, s, trace_slot(ctx, *kernels)));
-                Q(launch_tree_attention_mma(ctx->qkv, info, l * layer_elems, ctx->meta, n, c.n_head, cap, nullptr, nullptr, pdl, s, trace_slot(ctx, *kernels), ctx->attn_lo != 0, ctx->o8, sa, staged, attn_splits, attn_sms));
+                Q(launch_tree_attention_mma(ctx->qkv, info, l * layer_elems, ctx->meta, n, c.n_head, cap, nullptr, nullptr, pdl, s, trace_slot(ctx, *kernels), ctx->attn_lo != 0, ctx->o8, sa, attn_warps, attn_splits));
                 Q(gemm8(&t[1], &ssd_ctx::ActMaps::o_hi, ctx->x, d, L.b_o, d, d, grid8, L.s_o));
                 Q(launch_ln_prep(ctx->x, L.ln2_g, L.ln2_b, n, d, c.ln_eps, nullptr, nullptr, ctx->h, F, info, 0, pdl, s, trace_slot(ctx, *kernels), ctx->a8, sa));
                 Q(gemm8(&t[2], &ssd_ctx::ActMaps::a_hi, ctx->h, F, L.b_fc, d, F, grid8, L.s_fc));
@@ -377,7 +378,7 @@ cudaError_t enqueue_forward(ssd_ctx *ctx, int n, int cap, const NodeList &tk, co
             Q(launch_ln_prep(ctx->x, L.ln1_g, L.ln1_b, n, d, c.ln_eps, ctx->a_hi, a_lo, ctx->qkv, 3 * d, info, 0, pdl, s, trace_slot(ctx, *kernels)));
             Q(launch_gemm_ws(&t[0], &ag->a_hi, &ag->a_pair, ctx->qkv, info, 3 * d, L.b_qkv, n, d, 3 * d, lo, lgrid, sms, ctx->d_status, pdl, s, trace_slot(ctx, *kernels), nullptr, nullptr, 0, 4, gr));
             if (staged) Q(launch_kv_stage(ctx->qkv, info, l * layer_elems, n, c.n_head, cap, pdl, s, trace_slot(ctx, *kernels)));
-            Q(launch_tree_attention_mma(ctx->qkv, info, l * layer_elems, ctx->meta, n, c.n_head, cap, ctx->o_hi, o_lo, pdl, s, trace_slot(ctx, *kernels), ctx->attn_lo != 0, nullptr, 0, staged, attn_splits, attn_sms));
+            Q(launch_tree_attention_mma(ctx->qkv, info, l * layer_elems, ctx->meta, n, c.n_head, cap, ctx->o_hi, o_lo, pdl, s, trace_slot(ctx, *kernels), ctx->attn_lo != 0, nullptr, 0, attn_warps, attn_splits));
             Q(launch_gemm_ws(&t[1], &ag->o_hi, &ag->o_pair, ctx->x, info, d, L.b_o, n, d, d, lo, lgrid, sms, ctx->d_status, pdl, s, trace_slot(ctx, *kernels), nullptr, nullptr, 0, 4, gr));
             Q(launch_ln_prep(ctx->x, L.ln2_g, L.ln2_b, n, d, c.ln_eps, ctx->a_hi, a_lo, ctx->h, F, info, 0, pdl, s, trace_slot(ctx, *kernels)));
             Q(launch_gemm_ws(&t[2], &af->a_hi, &af->a_pair, ctx->h, info, F, L.b_fc, n, d, F, lo, lgrid, sms, ctx->d_status, pdl, s, trace_slot(ctx, *kernels), nullptr, nullptr, 0, 4, gr_fc));

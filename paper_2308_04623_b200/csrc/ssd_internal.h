@@ -153,7 +153,7 @@ cudaError_t tree_attention_mma_prepare();
 cudaError_t launch_tree_attention_mma(const float *qkv, const StepInfo *info, size_t layer_offset_elems, const TreeMeta &m, int n, int n_head,
                                       int cap, __nv_bfloat16 *o_hi, __nv_bfloat16 *o_lo, bool pdl, cudaStream_t s,
                                       unsigned long long *trace = nullptr, bool lo_pairs = true, uint8_t *planes8 = nullptr,
-                                      size_t plane_stride = 0, bool staged = false, int splits = 1, int sm_count = 0);
+                                      size_t plane_stride = 0, int staged_warps = 0, int splits = 1); // staged_warps: 0, or 4 / 8 warps per CTA reading the tree's rows from the cache
 // Writes the tree's K / V rows (bf16) to the cache's scratch slots and zeroes the rest of the last 16-key block; an attention launched
 // with `staged` then reads every block from the cache and stages nothing itself (worth its launch for large trees).
 cudaError_t launch_kv_stage(const float *qkv, const StepInfo *info, size_t layer_offset_elems, int n, int n_head, int cap, bool pdl, cudaStream_t s,
